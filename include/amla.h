@@ -1,0 +1,120 @@
+/*
+ * libamla -- paged MLA decode attention with exponent-add output rescaling (sm_100a).
+ *
+ * C ABI.  All pointers are borrowed; the library allocates no device memory and
+ * keeps no state between calls.  Work is enqueued on the caller's stream with no
+ * host synchronisation (sequence lengths are never read on the host).  Functions
+ * return an amla_status; nothing throws, aborts or prints.
+ *
+ * Shapes are those of the paper's decode setting (Section 3.1: G query rows of
+ * width D_k = 576 against a latent cache whose rows serve as K (576 columns) and,
+ * through their first D_v = 512 columns, as V; Section 2.2).  Paging, per-sequence
+ * lengths, the lse output, the causal rule between speculative query tokens and
+ * split-KV are additions the paper does not describe; they are defined below.
+ */
+#ifndef AMLA_H_
+#define AMLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  AMLA_OK = 0,
+  AMLA_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, misaligned buffer   */
+  AMLA_ERR_UNSUPPORTED = -2,    /* shape or device outside what the kernels cover       */
+  AMLA_ERR_WORKSPACE = -3,      /* workspace smaller than amla_mla_decode_workspace_size */
+  AMLA_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed                    */
+  AMLA_ERR_DEVICE_TIMEOUT = -5  /* a bounded device-side wait ran out (see amla_check_status) */
+} amla_status;
+
+/* Rescale variants, for A/B measurements (flags argument of amla_mla_decode_ex).
+ *   AMLA_RESCALE_ALG2 : Algorithm 2 as specified: P scaled by S16 = bf16(1/r_i), the accumulator
+ *                       updated by one INT32 add of N = dn*2^23 + round(2^23*(1.5*(c_i/c_{i-1}-1)+1e-6))
+ *                       (Lemma 3.1 + Appendix A).  Default.
+ *   AMLA_RESCALE_FOLD : Eq. 3 with 1/r_i folded exactly into the exponential's argument: the add is a
+ *                       pure exponent add dn*2^23 and is needed only when n_i changes.
+ *   AMLA_RESCALE_FMUL : Algorithm 1's FP32 multiply by exp(m_{i-1}-m_i) (the baseline the paper replaces).
+ * AMLA_FLAG_UNGUARDED_ADD uses the literal single integer add of Algorithm 2 line 14 (corrupts
+ * accumulators that are exactly 0.0 or below 2^-97; measurement only).
+ */
+enum {
+  AMLA_RESCALE_ALG2 = 0,
+  AMLA_RESCALE_FOLD = 1,
+  AMLA_RESCALE_FMUL = 2,
+  AMLA_RESCALE_MASK = 3,
+  AMLA_FLAG_UNGUARDED_ADD = 4,
+  AMLA_FLAG_KERNEL_SIMT = 8     /* run the scalar bring-up kernel instead of the tensor-core kernel */
+};
+
+/* Human-readable name of a status code (static storage). */
+const char* amla_status_string(int status);
+
+/* Bytes of device workspace amla_mla_decode needs for these sizes on `device`
+ * (its SM count bounds the number of KV splits).  Host-only; no CUDA work is enqueued. */
+int amla_mla_decode_workspace_size(int B, int Sq, int H, int max_blocks_per_seq, int device,
+                                   size_t* bytes_out);
+
+/*
+ * out[b,t,h,:] = softmax_j(scale * q[b,t,h,:] . k_j) @ k_j[0:512]   over the visible keys j of sequence b,
+ * lse[b,t,h]   = ln sum_j exp(scale * q[b,t,h,:] . k_j)                          (Eq. 1; Algorithm 2)
+ *
+ * Key j of sequence b is row (j % 64) of page block_table[b][j / 64] of kv_cache.  Query token t sees
+ * key j iff 0 <= j < seqlens[b] and j <= seqlens[b] - Sq + t (the Sq query tokens are the last Sq
+ * positions; each sees itself and everything before).  A row with no visible key gets out = 0,
+ * lse = -inf.
+ *
+ *   q            device, bf16 [B, Sq, H, 576], contiguous, 16-byte aligned
+ *   kv_cache     device, bf16 [num_blocks, 64, 576], contiguous, 16-byte aligned.  Rows of a used page
+ *                beyond the sequence length must hold finite values (they are multiplied by zero).
+ *   block_table  device, int32 [B, max_blocks_per_seq]; entries beyond ceil(seqlens[b]/64) are ignored
+ *   seqlens      device, int32 [B], 0 <= seqlens[b] <= 64 * max_blocks_per_seq
+ *   out          device, bf16 [B, Sq, H, 512], 16-byte aligned
+ *   lse          device, fp32 [B, Sq, H], natural logarithm
+ *   workspace    device, 256-byte aligned, at least amla_mla_decode_workspace_size() bytes; contents
+ *                need not be preserved or initialised; calls that overlap in time need distinct ones
+ *   cuda_stream  a cudaStream_t (NULL = default stream)
+ *
+ * Supported: 1 <= Sq <= 8, 1 <= H <= 128 with Sq*H a multiple of 128 or smaller than 128 ... any Sq*H
+ * up to 1024 rows; page size 64; sm_100 devices only (AMLA_ERR_UNSUPPORTED otherwise).
+ * Argument errors are reported before anything is launched.
+ */
+int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_table,
+                    const int32_t* seqlens, float softmax_scale, int B, int Sq, int H, int num_blocks,
+                    int max_blocks_per_seq, void* out, float* lse, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* Same, with a flags word selecting a rescale variant (see the enum above). */
+int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block_table,
+                       const int32_t* seqlens, float softmax_scale, int B, int Sq, int H,
+                       int num_blocks, int max_blocks_per_seq, void* out, float* lse, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream, int flags);
+
+/* Synchronises `cuda_stream` and reads the status word the kernels keep at the start of the
+ * workspace: AMLA_OK, or AMLA_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel expired (the
+ * kernel then returned early and the outputs are undefined).  Optional. */
+int amla_check_status(const void* workspace, void* cuda_stream);
+
+/* Number of kernels the most recent amla_mla_decode[_ex] call on this thread launched. */
+int amla_last_launch_count(void);
+
+/*
+ * Host mirror of the device-side split-KV schedule (the plan is not in the paper; it exists because
+ * B * ceil(Sq*H/128) work items are far fewer than the SMs).  Items are (sequence, 128-row block)
+ * pairs in order; their 64-key tiles form one linear range that is cut into num_parts equal parts.
+ * For every (part, item) intersection ("unit") one record of 6 int32 is written:
+ *   part, item, tile_begin, tile_end (within the item), slot (-1 = writes out/lse directly,
+ *   otherwise index of its fp32 partial), n_split of the item.
+ * seqlens is a HOST array here.  Returns the number of units, or a negative amla_status
+ * (AMLA_ERR_WORKSPACE if max_units is too small).
+ */
+int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int num_parts, int32_t* units,
+                   int max_units);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMLA_H_ */

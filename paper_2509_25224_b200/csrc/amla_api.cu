@@ -1,0 +1,223 @@
+// C-ABI entry points of libamla: argument validation, workspace carving and the three launches
+// (schedule prefix, decode, combine) on the caller's stream.
+#include <cstring>
+
+#include "../../include/amla.h"
+#include "amla_common.cuh"
+
+namespace amla {
+cudaError_t launch_plan(const DecodeParams& prm, int* prefix_out, cudaStream_t stream);
+cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream);
+cudaError_t launch_decode_simt(const DecodeParams& prm, cudaStream_t stream);
+// Returns cudaSuccess, or an error; sets *unsupported when the device cannot run the kernel.
+cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* unsupported);
+int decode_tc_parts(int sm_count);
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxRows = 1024;   // Sq * H
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+  size_t status_off, prefix_off, part_lse_off, part_o_off, total;
+};
+
+Layout make_layout(int n_items, int max_parts) {
+  Layout l;
+  l.status_off = 0;
+  l.prefix_off = kAlign;
+  l.part_lse_off = l.prefix_off + align_up(sizeof(int) * (static_cast<size_t>(n_items) + 1));
+  l.part_o_off = l.part_lse_off + align_up(sizeof(float) * 2 * static_cast<size_t>(max_parts) * kRowBlock);
+  l.total = l.part_o_off + sizeof(float) * 2 * static_cast<size_t>(max_parts) * kRowBlock * kDv;
+  return l;
+}
+
+int check_shape(int B, int Sq, int H, int max_blocks_per_seq) {
+  if (B <= 0 || Sq <= 0 || H <= 0 || max_blocks_per_seq <= 0) return AMLA_ERR_INVALID_ARG;
+  if (Sq > 8 || H > 128 || Sq * H > kMaxRows) return AMLA_ERR_UNSUPPORTED;
+  if (static_cast<long long>(max_blocks_per_seq) * kPage > (1ll << 30)) return AMLA_ERR_UNSUPPORTED;
+  if (static_cast<long long>(B) * ((Sq * H + kRowBlock - 1) / kRowBlock) > (1ll << 24)) return AMLA_ERR_UNSUPPORTED;
+  return AMLA_OK;
+}
+
+int sm_count_of(int device, int* sms, int* cc_major) {
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  *sms = prop.multiProcessorCount;
+  *cc_major = prop.major;
+  return AMLA_OK;
+}
+
+thread_local int g_last_launches = 0;
+
+}  // namespace
+}  // namespace amla
+
+using namespace amla;
+
+extern "C" const char* amla_status_string(int status) {
+  switch (status) {
+    case AMLA_OK: return "ok";
+    case AMLA_ERR_INVALID_ARG: return "invalid argument";
+    case AMLA_ERR_UNSUPPORTED: return "unsupported shape or device";
+    case AMLA_ERR_WORKSPACE: return "workspace too small";
+    case AMLA_ERR_CUDA: return "CUDA call failed";
+    case AMLA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int amla_mla_decode_workspace_size(int B, int Sq, int H, int max_blocks_per_seq, int device,
+                                              size_t* bytes_out) {
+  if (!bytes_out) return AMLA_ERR_INVALID_ARG;
+  int rc = check_shape(B, Sq, H, max_blocks_per_seq);
+  if (rc != AMLA_OK) return rc;
+  int sms = 0, cc = 0;
+  rc = sm_count_of(device, &sms, &cc);
+  if (rc != AMLA_OK) return rc;
+  const int nrb = (Sq * H + kRowBlock - 1) / kRowBlock;
+  *bytes_out = make_layout(B * nrb, sms).total;
+  return AMLA_OK;
+}
+
+extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block_table,
+                                  const int32_t* seqlens, float softmax_scale, int B, int Sq, int H,
+                                  int num_blocks, int max_blocks_per_seq, void* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream, int flags) {
+  g_last_launches = 0;
+  if (!q || !kv_cache || !block_table || !seqlens || !out || !lse || !workspace) return AMLA_ERR_INVALID_ARG;
+  if (num_blocks <= 0 || !(softmax_scale == softmax_scale)) return AMLA_ERR_INVALID_ARG;
+  int rc = check_shape(B, Sq, H, max_blocks_per_seq);
+  if (rc != AMLA_OK) return rc;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kv_cache) | reinterpret_cast<uintptr_t>(out)) & 15)
+    return AMLA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(block_table) | reinterpret_cast<uintptr_t>(seqlens) | reinterpret_cast<uintptr_t>(lse)) & 3)
+    return AMLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) return AMLA_ERR_INVALID_ARG;
+  if ((flags & AMLA_RESCALE_MASK) == 3) return AMLA_ERR_INVALID_ARG;
+
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  int sms = 0, cc = 0;
+  rc = sm_count_of(device, &sms, &cc);
+  if (rc != AMLA_OK) return rc;
+  if (cc != 10) return AMLA_ERR_UNSUPPORTED;
+
+  const int nrb = (Sq * H + kRowBlock - 1) / kRowBlock;
+  const int n_items = B * nrb;
+  const Layout lay = make_layout(n_items, sms);
+  if (workspace_bytes < lay.total) return AMLA_ERR_WORKSPACE;
+
+  char* ws = static_cast<char*>(workspace);
+  DecodeParams prm;
+  std::memset(&prm, 0, sizeof(prm));
+  prm.q = static_cast<const __nv_bfloat16*>(q);
+  prm.kv = static_cast<const __nv_bfloat16*>(kv_cache);
+  prm.block_table = block_table;
+  prm.seqlens = seqlens;
+  prm.out = static_cast<__nv_bfloat16*>(out);
+  prm.lse = lse;
+  prm.status = reinterpret_cast<int*>(ws + lay.status_off);
+  int* prefix = reinterpret_cast<int*>(ws + lay.prefix_off);
+  prm.prefix = prefix;
+  prm.part_lse = reinterpret_cast<float*>(ws + lay.part_lse_off);
+  prm.part_o = reinterpret_cast<float*>(ws + lay.part_o_off);
+  prm.scale_log2 = softmax_scale * kLog2e;
+  prm.B = B; prm.Sq = Sq; prm.H = H;
+  prm.R = Sq * H;
+  prm.nrb = nrb;
+  prm.n_items = n_items;
+  prm.num_blocks = num_blocks;
+  prm.max_blocks_per_seq = max_blocks_per_seq;
+  prm.flags = flags;
+  const bool simt = (flags & AMLA_FLAG_KERNEL_SIMT) != 0;
+  prm.P = simt ? sms : decode_tc_parts(sms);
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  ++g_last_launches;
+  if (simt) {
+    if (launch_decode_simt(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  } else {
+    int unsupported = 0;
+    if (launch_decode_tc(prm, stream, &unsupported) != cudaSuccess) {
+      cudaGetLastError();
+      return unsupported ? AMLA_ERR_UNSUPPORTED : AMLA_ERR_CUDA;
+    }
+  }
+  ++g_last_launches;
+  if (launch_combine(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  ++g_last_launches;
+  return AMLA_OK;
+}
+
+extern "C" int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_table,
+                               const int32_t* seqlens, float softmax_scale, int B, int Sq, int H,
+                               int num_blocks, int max_blocks_per_seq, void* out, float* lse,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return amla_mla_decode_ex(q, kv_cache, block_table, seqlens, softmax_scale, B, Sq, H, num_blocks,
+                            max_blocks_per_seq, out, lse, workspace, workspace_bytes, cuda_stream,
+                            AMLA_RESCALE_ALG2);
+}
+
+extern "C" int amla_check_status(const void* workspace, void* cuda_stream) {
+  if (!workspace) return AMLA_ERR_INVALID_ARG;
+  int st = 0;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
+    cudaGetLastError();
+    return AMLA_ERR_CUDA;
+  }
+  return st == kStatusOk ? AMLA_OK : AMLA_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" int amla_last_launch_count(void) { return g_last_launches; }
+
+extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int num_parts, int32_t* units,
+                              int max_units) {
+  if (!seqlens || !units || num_parts <= 0 || max_units < 0) return AMLA_ERR_INVALID_ARG;
+  int rc = check_shape(B, Sq, H, 1);
+  if (rc != AMLA_OK) return rc;
+  const int nrb = (Sq * H + kRowBlock - 1) / kRowBlock;
+  const int n_items = B * nrb;
+  int* prefix = new int[n_items + 1];
+  int acc = 0;
+  for (int it = 0; it < n_items; ++it) {
+    prefix[it] = acc;
+    int n = seqlens[it / nrb];
+    if (n < 0) n = 0;
+    acc += (n + kPage - 1) / kPage;
+  }
+  prefix[n_items] = acc;
+  const Plan plan = Plan::make(prefix, n_items, num_parts);
+  int n_units = 0;
+  bool overflow = false;
+  if (acc > 0) {
+    for (int p = 0; p < plan.P; ++p) {
+      const int g0 = plan.part_start(p), g1 = plan.part_start(p + 1);
+      int g = g0;
+      while (g < g1) {
+        const int it = plan.item_of_tile(g);
+        const int a = prefix[it], e = prefix[it + 1];
+        const int t0 = g - a, t1 = (e < g1 ? e : g1) - a;
+        g = a + t1;
+        int p_first, p_last;
+        const int nsplit = plan.item_parts(it, &p_first, &p_last);
+        if (n_units < max_units) {
+          int32_t* u = units + 6 * n_units;
+          u[0] = p; u[1] = it; u[2] = t0; u[3] = t1;
+          u[4] = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
+          u[5] = nsplit;
+        } else {
+          overflow = true;
+        }
+        ++n_units;
+      }
+    }
+  }
+  delete[] prefix;
+  return overflow ? AMLA_ERR_WORKSPACE : n_units;
+}

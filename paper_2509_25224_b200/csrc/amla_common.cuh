@@ -1,0 +1,192 @@
+// Shared definitions of the libamla kernels: problem constants, the parameter block, the split-KV
+// schedule arithmetic (host + device), and the per-row scalar recurrence of Algorithm 2.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace amla {
+
+constexpr int kDqk = 576;      // K width: 512 latent + 64 RoPE columns (Section 3.1)
+constexpr int kDv = 512;       // V width: the latent columns
+constexpr int kPage = 64;      // keys per cache page == keys per tile
+constexpr int kRowBlock = 128; // query rows per work item (= MMA M)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Status word kept at workspace[0].
+constexpr int kStatusOk = 0;
+constexpr int kStatusTimeout = 1;
+
+struct DecodeParams {
+  const __nv_bfloat16* q;        // [B, Sq, H, 576] == [B, R, 576]
+  const __nv_bfloat16* kv;       // [num_blocks, 64, 576]
+  const int32_t* block_table;    // [B, max_blocks_per_seq]
+  const int32_t* seqlens;        // [B]
+  __nv_bfloat16* out;            // [B, R, 512]
+  float* lse;                    // [B, R]
+  int* status;                   // workspace status word
+  const int* prefix;             // [n_items + 1] linear tile index of each item's first tile
+  float* part_o;                 // [2 * P, 128, 512] fp32 normalised partial outputs
+  float* part_lse;               // [2 * P, 128]      partial lse (natural log)
+  float scale_log2;              // softmax_scale * log2(e)
+  int B, Sq, H;
+  int R;                         // Sq * H query rows per sequence
+  int nrb;                       // row blocks per sequence = ceil(R / 128)
+  int n_items;                   // B * nrb
+  int num_blocks, max_blocks_per_seq;
+  int P;                         // parts the linear tile range is cut into
+  int flags;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Split-KV schedule.  Items (sequence b, row block rb) in order it = b * nrb + rb own
+// ceil(N_b / 64) tiles each; prefix[it] is the linear index of an item's first tile and
+// L = prefix[n_items] the total.  Part p owns linear tiles [p*L/P, (p+1)*L/P).
+// ---------------------------------------------------------------------------------------------
+struct Plan {
+  const int* prefix;
+  int n_items;
+  int L;
+  int P;
+
+  // With fewer tiles than parts only the first L parts get work (one tile each).
+  __host__ __device__ static Plan make(const int* prefix, int n_items, int max_parts) {
+    Plan pl;
+    pl.prefix = prefix;
+    pl.n_items = n_items;
+    pl.L = prefix[n_items];
+    pl.P = pl.L < max_parts ? (pl.L > 0 ? pl.L : 1) : max_parts;
+    return pl;
+  }
+  __host__ __device__ int part_start(int p) const {
+    if (p >= P) return L;
+    return static_cast<int>((static_cast<long long>(p) * L) / P);
+  }
+  __host__ __device__ int part_of_tile(int g) const {
+    int p = static_cast<int>((static_cast<long long>(g) * P) / L);
+    if (p > P - 1) p = P - 1;
+    while (p + 1 < P && part_start(p + 1) <= g) ++p;
+    while (p > 0 && part_start(p) > g) --p;
+    return p;
+  }
+  // Largest item index whose first tile is <= g (zero-tile items are skipped automatically).
+  __host__ __device__ int item_of_tile(int g) const {
+    int lo = 0, hi = n_items - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (prefix[mid] <= g) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+  }
+  // Parts [p_first, p_last] that touch item `it`; returns the split count (0 for an empty item).
+  __host__ __device__ int item_parts(int it, int* p_first, int* p_last) const {
+    const int a = prefix[it], e = prefix[it + 1];
+    if (e <= a) { *p_first = 0; *p_last = -1; return 0; }
+    *p_first = part_of_tile(a);
+    *p_last = part_of_tile(e - 1);
+    return *p_last - *p_first + 1;
+  }
+  // Partial slot of the unit (part p, item it): a part has at most two partial units, the one that
+  // began in an earlier part / begins exactly at the part start (slot 2p) and a later one (2p+1).
+  __host__ __device__ int slot_of(int p, int it, int p_first) const {
+    return 2 * p + ((p == p_first && prefix[it] > part_start(p)) ? 1 : 0);
+  }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Lemma 3.1: F * 2^n == AS_FP32(AS_INT32(F) + n * 2^23) for normal F and 0 < E + n < 255.
+// The guarded form adds to the magnitude bits and clamps at zero, so exact zeros stay zero and
+// values that would fall below the normal range become zero/denormal instead of wrapping.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float exponent_add_guarded(float f, int n_bits) {
+  const int i = __float_as_int(f);
+  const int mag = max((i & 0x7fffffff) + n_bits, 0);
+  return __int_as_float(mag | (i & 0x80000000));
+}
+__device__ __forceinline__ float exponent_add_raw(float f, int n_bits) {
+  return __int_as_float(__float_as_int(f) + n_bits);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float bf16_round(float x) {
+  return __bfloat162float(__float2bfloat16_rn(x));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Per-row running state and the scalar part of one tile step, in the base-2 domain:
+// a_j = s_j * log2(e), so exp(s_j - m) = 2^(a_j - m2) and n_i = round(-m_i / ln 2) = round(-m2).
+// ---------------------------------------------------------------------------------------------
+struct RowState {
+  float m2;      // running max of a_j (-inf before the first visible key)
+  float l;       // running row sum of P (unscaled FP32, Algorithm 2 line 6)
+  float n;       // n_i of the last tile with a visible key
+  float c;       // c_i of that tile (Appendix A: r_i / r'_i = S16 / S32)
+  float s_out;   // scale folded into P for that tile (S16, S32 or 1 depending on the mode)
+  int started;   // the row's accumulator has received a P V product
+};
+
+__device__ __forceinline__ void row_state_init(RowState& st) {
+  st.m2 = -INFINITY; st.l = 0.f; st.n = 0.f; st.c = 1.f; st.s_out = 1.f; st.started = 0;
+}
+
+// Result of the scalar step for one row and one tile.
+struct RowStep {
+  float m2_sub;   // value to subtract inside the exponential (0 when the row has no visible key yet)
+  float p_scale;  // factor folded into P before the bf16 cast
+  float l_up;     // exp2(m2_old - m2_new), multiplies the old row sum (and the old O in FMUL mode)
+  int n_bits;     // integer added to the accumulator's bit pattern (0 = leave the row alone)
+};
+
+// mode: 0 = Algorithm 2, 1 = exact fold (Eq. 3), 2 = FP32 multiply (Algorithm 1).
+template <int kMode>
+__device__ __forceinline__ RowStep row_step(RowState& st, float tile_max2) {
+  RowStep r;
+  const float m_old = st.m2;
+  const float m_new = fmaxf(m_old, tile_max2);
+  if (m_new == -INFINITY) {        // nothing visible so far: P will be all zeros
+    r.m2_sub = 0.f; r.p_scale = 1.f; r.l_up = 1.f; r.n_bits = 0;
+    return r;
+  }
+  r.m2_sub = m_new;
+  r.l_up = (m_old == -INFINITY) ? 0.f : ex2_approx(m_old - m_new);
+  r.n_bits = 0;
+  if (kMode == 2) {
+    r.p_scale = 1.f;
+    st.s_out = 1.f;
+  } else {
+    const float n_i = rintf(-m_new);                       // Alg. 2 line 6
+    const float s32 = ex2_approx(n_i + m_new);             // line 7: 1/r_i in [1/sqrt2, sqrt2]
+    if (kMode == 0) {
+      const float s16 = bf16_round(s32);                   // line 8
+      const float c_i = __fdividef(s16, s32);              // Appendix A: c_i = r_i / r'_i
+      if (st.started && m_new != m_old) {
+        const float eps = 1.5f * (__fdividef(c_i, st.c) - 1.f);           // line 9
+        const int dn = static_cast<int>(fmaxf(n_i - st.n, -30.f));        // line 11
+        r.n_bits = dn * (1 << 23) + __float2int_rn((eps + 1e-6f) * 8388608.f);   // line 12
+      }
+      st.c = c_i;
+      r.p_scale = s16;                                     // line 10
+      st.s_out = s16;
+    } else {
+      if (st.started && n_i != st.n) {
+        const int dn = static_cast<int>(fmaxf(n_i - st.n, -30.f));
+        r.n_bits = dn * (1 << 23);
+      }
+      r.p_scale = s32;
+      st.s_out = s32;
+    }
+    st.n = n_i;
+  }
+  st.m2 = m_new;
+  st.started = 1;
+  return r;
+}
+
+}  // namespace amla

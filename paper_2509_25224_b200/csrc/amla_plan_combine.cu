@@ -1,0 +1,131 @@
+// Split-KV schedule (prefix of tile counts per work item) and the lse-weighted combine of split
+// partials.  Neither is in the paper: its kernel runs batch 96 on 48 cores, whereas a decode batch
+// here has far fewer (sequence, row-block) items than the GPU has SMs.  The combine is the
+// log-sum-exp merge that follows from the blockwise associativity of Algorithm 1's recurrence.
+#include "amla_common.cuh"
+
+namespace amla {
+
+// One block.  prefix[it] = sum over items before `it` of ceil(seqlens[b(it)] / 64); also resets the
+// status word.  n_items is small (B * ceil(Sq*H/128)); a chunked block scan covers any size.
+__global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_items,
+                            int* __restrict__ prefix, int* __restrict__ status) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) { carry = 0; *status = kStatusOk; }
+  __syncthreads();
+  for (int base = 0; base < n_items; base += blockDim.x) {
+    const int it = base + tid;
+    int v = 0;
+    if (it < n_items) {
+      int n = seqlens[it / nrb];
+      n = n < 0 ? 0 : n;
+      v = (n + kPage - 1) / kPage;
+    }
+    int x = v;  // inclusive warp scan
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
+    }
+    if (lane == 31) warp_sums[wid] = x;
+    __syncthreads();
+    if (wid == 0) {
+      int s = (lane < (blockDim.x >> 5)) ? warp_sums[lane] : 0;
+      for (int o = 1; o < 32; o <<= 1) {
+        int y = __shfl_up_sync(0xffffffffu, s, o);
+        if (lane >= o) s += y;
+      }
+      warp_sums[lane] = s;  // inclusive over warps
+    }
+    __syncthreads();
+    const int before = carry + (wid ? warp_sums[wid - 1] : 0) + (x - v);
+    if (it < n_items) prefix[it] = before;
+    __syncthreads();
+    if (tid == blockDim.x - 1) carry = before + v;
+    __syncthreads();
+  }
+  if (tid == 0) prefix[n_items] = carry;
+}
+
+// One warp per query row.  Items that one part covered entirely were written by the decode kernel
+// and are skipped; items without tiles get out = 0, lse = -inf; split items are merged:
+//   lse = ln sum_s exp(lse_s),  out = sum_s exp(lse_s - lse) * out_s.
+__global__ void combine_kernel(DecodeParams prm) {
+  const int warps_per_block = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int row_global = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  const int rows_padded = prm.nrb * kRowBlock;
+  const int b = row_global / rows_padded;
+  if (b >= prm.B) return;
+  const int rin = row_global - b * rows_padded;   // row within the sequence, padded to row blocks
+  if (rin >= prm.R) return;
+  const int rb = rin / kRowBlock, rr = rin % kRowBlock;
+  const int it = b * prm.nrb + rb;
+
+  const Plan plan = Plan::make(prm.prefix, prm.n_items, prm.P);
+  int p_first, p_last;
+  const int nsplit = plan.L > 0 ? plan.item_parts(it, &p_first, &p_last) : 0;
+  if (nsplit == 1) return;
+
+  __nv_bfloat16* orow = prm.out + (static_cast<size_t>(b) * prm.R + rin) * kDv;
+  float* lrow = prm.lse + static_cast<size_t>(b) * prm.R + rin;
+  if (nsplit == 0) {
+    for (int c = lane * 8; c < kDv; c += 32 * 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
+    if (lane == 0) *lrow = -INFINITY;
+    return;
+  }
+  float mx = -INFINITY;
+  for (int p = p_first; p <= p_last; ++p) {
+    const int slot = plan.slot_of(p, it, p_first);
+    mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(slot) * kRowBlock + rr]);
+  }
+  if (mx == -INFINITY) {   // no split saw a visible key for this row
+    for (int c = lane * 8; c < kDv; c += 32 * 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
+    if (lane == 0) *lrow = -INFINITY;
+    return;
+  }
+  float acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+  float tot = 0.f;
+  for (int p = p_first; p <= p_last; ++p) {
+    const int slot = plan.slot_of(p, it, p_first);
+    const float ls = prm.part_lse[static_cast<size_t>(slot) * kRowBlock + rr];
+    const float w = expf(ls - mx);   // 0 for a split that saw nothing (lse_s = -inf)
+    tot += w;
+    const float* src = prm.part_o + (static_cast<size_t>(slot) * kRowBlock + rr) * kDv;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 v = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
+      acc[4 * i + 0] += w * v.x; acc[4 * i + 1] += w * v.y;
+      acc[4 * i + 2] += w * v.z; acc[4 * i + 3] += w * v.w;
+    }
+  }
+  const float inv = 1.f / tot;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc[4 * i + 0] * inv, acc[4 * i + 1] * inv);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc[4 * i + 2] * inv, acc[4 * i + 3] * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(orow + i * 128 + lane * 4) = pk;
+  }
+  if (lane == 0) *lrow = mx + logf(tot);
+}
+
+cudaError_t launch_plan(const DecodeParams& prm, int* prefix_out, cudaStream_t stream) {
+  plan_kernel<<<1, 1024, 0, stream>>>(prm.seqlens, prm.nrb, prm.n_items, prefix_out, prm.status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream) {
+  const int warps_per_block = 8;
+  const long rows = static_cast<long>(prm.B) * prm.nrb * kRowBlock;
+  const int blocks = static_cast<int>((rows + warps_per_block - 1) / warps_per_block);
+  combine_kernel<<<blocks, warps_per_block * 32, 0, stream>>>(prm);
+  return cudaGetLastError();
+}
+
+}  // namespace amla
