@@ -1,6 +1,550 @@
-// placeholder
+// Tensor-core MLA decode kernel for sm_100a.
+//
+// A cluster of two CTAs works on one 128-row block of query rows and a range of 64-key tiles:
+//
+//   score CTA (cluster rank 0)   Q (128 x 576 bf16) resident in tensor memory as the A operand;
+//       K tiles streamed by TMA; S = Q K^T by tcgen05.mma into a double-buffered TMEM tile; the
+//       softmax warpgroup runs Algorithm 2's per-row recurrence (lines 5-12) and writes the bf16
+//       probabilities P~ = bf16(P * S16) and the per-row integer N into the value CTA's shared
+//       memory (distributed shared memory).
+//   value CTA (cluster rank 1)   the whole FP32 accumulator O (128 x 512) lives in its tensor memory;
+//       V tiles (first 512 columns of the same cache rows) streamed by TMA; a correction warpgroup
+//       applies N to the bit patterns of O (lines 13-16; Lemma 3.1) for rows whose maximum moved,
+//       then O += P~ V by tcgen05.mma (lines 17-18); the epilogue divides by l * S16 (line 20).
+//
+// This is the counterpart of the paper's split between matrix and vector units (Section 3.3) with
+// its [C1, C2, V1] steady-state order (Section 4.1): QK^T of tile i+1 is issued before P V of tile i
+// finishes, and the softmax of tile i+1 overlaps both.  What differs: O never leaves tensor memory,
+// so the integer add is a TMEM load/add/store rather than an atomic in global memory.
+//
+// All waits are bounded; on expiry the kernel records kStatusTimeout and unwinds.
 #include "amla_common.cuh"
+#include "amla_sm100.cuh"
+
 namespace amla {
-int decode_tc_parts(int sm_count) { return sm_count / 2; }
-cudaError_t launch_decode_tc(const DecodeParams&, cudaStream_t, int* unsupported) { *unsupported = 1; return cudaErrorNotSupported; }
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kThreads = 224;            // warps 0-3: softmax / correction, 4: TMA, 5: MMA + TMEM alloc, 6: relay
+constexpr int kNumKStages = 3;
+constexpr int kNumVStages = 2;
+constexpr uint32_t kBoxBytes = 64 * 64 * 2;             // one 64-key x 64-column TMA box
+constexpr uint32_t kKStageBytes = 9 * kBoxBytes;        // 73728
+constexpr uint32_t kVStageBytes = 8 * kBoxBytes;        // 65536
+constexpr uint32_t kPBytes = 128 * 64 * 2;              // 16384
+
+// tensor-memory columns
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kQCol = 0;            // score CTA: Q, 288 columns (two bf16 per column)
+constexpr uint32_t kSCol = 288;          // score CTA: S buffers, 2 x 64 columns
+// value CTA: O occupies columns 0..511
+
+// shared-memory layout (offsets from the 1024-aligned base); both CTAs allocate the larger of the two
+constexpr uint32_t kOffK = 0;                                          // score CTA
+constexpr uint32_t kOffABars = kNumKStages * kKStageBytes;             // 221184
+constexpr uint32_t kOffV = 0;                                          // value CTA
+constexpr uint32_t kOffP = kNumVStages * kVStageBytes;                 // 131072
+constexpr uint32_t kOffN = kOffP + 2 * kPBytes;                        // int32 [2][128]
+constexpr uint32_t kOffFin = kOffN + 2 * 128 * 4;                      // float2 [2][128] (1/(l*S16), lse)
+constexpr uint32_t kOffBBars = kOffFin + 2 * 128 * 8;
+constexpr uint32_t kBarBytes = 256;
+constexpr uint32_t kSmemA = kOffABars + kBarBytes;
+constexpr uint32_t kSmemB = kOffBBars + kBarBytes;
+constexpr uint32_t kSmemBytes = (kSmemA > kSmemB ? kSmemA : kSmemB) + 1024;
+
+// barrier indices, score CTA
+enum { A_KFULL = 0, A_KEMPTY = A_KFULL + kNumKStages, A_SFULL = A_KEMPTY + kNumKStages, A_SEMPTY = A_SFULL + 2,
+       A_PEMPTY = A_SEMPTY + 2, A_QREADY = A_PEMPTY + 2, A_QFREE, A_NUM };
+// barrier indices, value CTA
+enum { B_VFULL = 0, B_VEMPTY = B_VFULL + kNumVStages, B_PFULL = B_VEMPTY + kNumVStages, B_OREADY = B_PFULL + 2,
+       B_PVDONE = B_OREADY + 2, B_FINFULL = B_PVDONE + 2, B_NUM = B_FINFULL + 2 };
+static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
+
+struct Unit {
+  int b, r0, nrows, n_b, t0, t1, slot;
+};
+
+// Walks the (part, item) intersections of this cluster's part in schedule order.
+struct UnitIter {
+  const DecodeParams& prm;
+  Plan plan;
+  int p, g, g1;
+  __device__ UnitIter(const DecodeParams& prm_, int part) : prm(prm_), plan(Plan::make(prm_.prefix, prm_.n_items, prm_.P)), p(part) {
+    if (plan.L <= 0 || p >= plan.P) { g = g1 = 0; }
+    else { g = plan.part_start(p); g1 = plan.part_start(p + 1); }
+  }
+  __device__ bool next(Unit& u) {
+    if (g >= g1) return false;
+    const int it = plan.item_of_tile(g);
+    const int a = prm.prefix[it], e = prm.prefix[it + 1];
+    u.t0 = g - a;
+    u.t1 = min(e, g1) - a;
+    g = a + u.t1;
+    u.b = it / prm.nrb;
+    u.r0 = (it % prm.nrb) * kRowBlock;
+    u.nrows = min(kRowBlock, prm.R - u.r0);
+    u.n_b = min(max(prm.seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
+    int p_first, p_last;
+    const int nsplit = plan.item_parts(it, &p_first, &p_last);
+    u.slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
+    return true;
+  }
+};
+
+__device__ __forceinline__ void report_timeout(int* status) { atomicExch(status, kStatusTimeout); }
+
+}  // namespace
+
+template <int kMode, bool kGuard>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool is_score = rank == 0;
+  const int part = blockIdx.x >> 1;
+
+  const uint32_t bars = smem_base + (is_score ? kOffABars : kOffBBars);
+  auto bar = [&](int i) { return bars + 8u * i; };
+  const uint32_t tmem_slot = bars + kBarBytes - 8;
+  // addresses of the peer's barriers / buffers (same dynamic-smem base in both CTAs)
+  const uint32_t peerA_bars = map_to_cta(smem_base + kOffABars, 0);
+  const uint32_t peerB_bars = map_to_cta(smem_base + kOffBBars, 1);
+  const uint32_t peerB_base = map_to_cta(smem_base, 1);
+
+  if (tid == 0) {
+    if (is_score) {
+      for (int i = 0; i < kNumKStages; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
+      for (int i = 0; i < 2; ++i) { mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 128); mbar_init(bar(A_PEMPTY + i), 1); }
+      mbar_init(bar(A_QREADY), 128);
+      mbar_init(bar(A_QFREE), 1);
+    } else {
+      for (int i = 0; i < kNumVStages; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(bar(B_PFULL + i), 128); mbar_init(bar(B_OREADY + i), 128);
+        mbar_init(bar(B_PVDONE + i), 1); mbar_init(bar(B_FINFULL + i), 128);
+      }
+    }
+    fence_mbar_init();
+    prefetch_tensormap(&kv_map);
+  }
+  if (wid == 5) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();          // peer barriers are initialised before anyone signals them
+  tc_fence_after_sync();
+  uint32_t tbase;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tbase) : "r"(tmem_slot));
+
+  bool ok = true;
+  UnitIter iter(prm, part);
+  Unit u;
+  uint32_t gt = 0;      // tiles processed by this cluster so far (all roles count identically)
+  uint32_t un = 0;      // units processed so far
+
+  if (is_score) {
+    // ======================================================================= score CTA
+    if (wid < 4) {
+      // ---- softmax warpgroup: thread = query row
+      const int r = tid;
+      const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+      while (ok && iter.next(u)) {
+        // Q row -> tensor memory (previous unit's QK^T must be finished with it)
+        ok = mbar_wait(bar(A_QFREE), (un & 1) ^ 1);
+        if (!ok) break;
+        tc_fence_after_sync();
+        {
+          const bool valid = r < u.nrows;
+          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDqk);
+#pragma unroll 1
+          for (int blk = 0; blk < 9; ++blk) {
+            uint32_t regs[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              uint4 v = valid ? __ldg(qrow + blk * 8 + c) : make_uint4(0, 0, 0, 0);
+              regs[4 * c] = v.x; regs[4 * c + 1] = v.y; regs[4 * c + 2] = v.z; regs[4 * c + 3] = v.w;
+            }
+            tmem_st_32x32b_x32(tbase + lane_base + kQCol + blk * 32, regs);
+          }
+          tmem_wait_st();
+        }
+        tc_fence_before_sync();
+        mbar_arrive(bar(A_QREADY));
+
+        RowState st;
+        row_state_init(st);
+        const int tok = (u.r0 + r) / prm.H;
+        const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);   // keys 0..visible-1 are seen by this row
+        const int first_masked_tile = (u.n_b - prm.Sq + 1) / kPage;  // tiles from here on may hold hidden keys
+
+        for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
+          const uint32_t s = gt & 1, k = gt >> 1;
+          ok = mbar_wait(bar(A_SFULL + s), k & 1);
+          if (!ok) break;
+          tc_fence_after_sync();
+          uint32_t a[64];
+          {
+            uint32_t lo[32], hi[32];
+            tmem_ld_32x32b_x32(tbase + lane_base + kSCol + 64 * s, lo);
+            tmem_ld_32x32b_x32(tbase + lane_base + kSCol + 64 * s + 32, hi);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) { a[i] = lo[i]; a[32 + i] = hi[i]; }
+          }
+          tc_fence_before_sync();
+          mbar_arrive(bar(A_SEMPTY + s));
+
+          // lines 5-6: scale, mask, running max
+          float tmax = -INFINITY;
+          if (t >= first_masked_tile || t < 0) {
+            const int jbase = t * kPage;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+              float v = __uint_as_float(a[i]) * prm.scale_log2;
+              v = (jbase + i < visible) ? v : -INFINITY;
+              a[i] = __float_as_uint(v);
+              tmax = fmaxf(tmax, v);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+              const float v = __uint_as_float(a[i]) * prm.scale_log2;
+              a[i] = __float_as_uint(v);
+              tmax = fmaxf(tmax, v);
+            }
+          }
+          const RowStep sp = row_step<kMode>(st, tmax);
+          // lines 6, 10: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
+          float rs = 0.f;
+          uint32_t pk[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float p0 = ex2_approx(__uint_as_float(a[2 * i]) - sp.m2_sub);
+            const float p1 = ex2_approx(__uint_as_float(a[2 * i + 1]) - sp.m2_sub);
+            rs += p0 + p1;
+            pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+          }
+          st.l = st.l * sp.l_up + rs;
+
+          // hand P~ and N to the value CTA
+          ok = mbar_wait(bar(A_PEMPTY + s), (k & 1) ^ 1);
+          if (!ok) break;
+          const uint32_t pdst = peerB_base + kOffP + s * kPBytes;
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            st_cluster_v4(pdst + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+          const uint32_t nword = (kMode == 2) ? __float_as_uint(sp.l_up) : static_cast<uint32_t>(sp.n_bits);
+          st_cluster_b32(peerB_base + kOffN + (s * 128 + r) * 4, nword);
+          fence_proxy_async_all();
+          mbar_arrive_cluster(peerB_bars + 8u * (B_PFULL + s));
+        }
+        if (!ok) break;
+        // line 20 scalars: 1 / (l * S16) and lse = m + ln l
+        {
+          const bool live = st.l > 0.f;
+          const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
+          const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
+          const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;
+          st_cluster_b32(fdst, __float_as_uint(inv));
+          st_cluster_b32(fdst + 4, __float_as_uint(lse));
+          mbar_arrive_cluster(peerB_bars + 8u * (B_FINFULL + (un & 1)));
+        }
+        ++un;
+      }
+      if (!ok) report_timeout(prm.status);
+    } else if (wid == 4) {
+      // ---- TMA producer: K tiles (all 576 columns)
+      if (lane == 0) {
+        uint32_t issued = 0;
+        while (ok && iter.next(u)) {
+          const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            const uint32_t stg = gt % kNumKStages, rnd = gt / kNumKStages;
+            ok = mbar_wait(bar(A_KEMPTY + stg), (rnd & 1) ^ 1);
+            if (!ok) break;
+            const int page = __ldg(bt + t);
+            mbar_arrive_expect_tx(bar(A_KFULL + stg), kKStageBytes);
+            const uint32_t dst = smem_base + kOffK + stg * kKStageBytes;
+#pragma unroll
+            for (int c = 0; c < 9; ++c) tma_load_2d(dst + c * kBoxBytes, &kv_map, c * 64, page * kPage, bar(A_KFULL + stg));
+            ++issued;
+          }
+        }
+        if (!ok) {
+          report_timeout(prm.status);
+          // let copies that are still in flight land before the CTA exits
+          for (uint32_t i = 0; i < kNumKStages && i < issued; ++i) {
+            const uint32_t n = issued - 1 - i;
+            mbar_wait(bar(A_KFULL + n % kNumKStages), (n / kNumKStages) & 1);
+          }
+        }
+      }
+    } else if (wid == 5) {
+      // ---- MMA issuer: S[s] = Q K_t^T, 36 steps of K = 16
+      if (lane == 0) {
+        constexpr uint32_t idesc = make_idesc_bf16(128, 64, false, false);
+        while (ok && iter.next(u)) {
+          ok = mbar_wait(bar(A_QREADY), un & 1);
+          if (!ok) break;
+          tc_fence_after_sync();
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            const uint32_t stg = gt % kNumKStages, rnd = gt / kNumKStages;
+            const uint32_t s = gt & 1, k = gt >> 1;
+            ok = mbar_wait(bar(A_KFULL + stg), rnd & 1);
+            if (!ok) break;
+            ok = mbar_wait(bar(A_SEMPTY + s), (k & 1) ^ 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t kbase = smem_base + kOffK + stg * kKStageBytes;
+            const uint32_t d = tbase + kSCol + 64 * s;
+#pragma unroll
+            for (int ks = 0; ks < 36; ++ks) {
+              const uint64_t bd = make_smem_desc_sw128(kbase + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024);
+              mma_ts(d, tbase + kQCol + 8 * ks, bd, idesc, ks > 0);
+            }
+            mma_commit(bar(A_KEMPTY + stg));
+            mma_commit(bar(A_SFULL + s));
+          }
+          if (!ok) break;
+          mma_commit(bar(A_QFREE));
+          ++un;
+        }
+        if (!ok) report_timeout(prm.status);
+      }
+    }
+  } else {
+    // ======================================================================= value CTA
+    if (wid < 4) {
+      // ---- correction + epilogue warpgroup: thread = query row
+      const int r = tid;
+      const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+      while (ok && iter.next(u)) {
+        for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
+          const uint32_t s = gt & 1, k = gt >> 1;
+          ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
+          if (!ok) break;
+          uint32_t nword;
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(nword) : "r"(smem_base + kOffN + (s * 128 + r) * 4));
+          const bool mine = (kMode == 2) ? (__uint_as_float(nword) != 1.f) : (nword != 0u);
+          if (__any_sync(0xffffffffu, mine) && t > u.t0) {
+            // lines 13-16: O <- AS_FP32(AS_INT32(O) + N), after P V of the previous tile has landed
+            const uint32_t gp = gt - 1;
+            ok = mbar_wait(bar(B_PVDONE + (gp & 1)), (gp >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 16; ++c) {
+              uint32_t o[32];
+              tmem_ld_32x32b_x32(tbase + lane_base + 32 * c, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                float f = __uint_as_float(o[i]);
+                if (kMode == 2) f *= __uint_as_float(nword);
+                else f = kGuard ? exponent_add_guarded(f, static_cast<int>(nword)) : exponent_add_raw(f, static_cast<int>(nword));
+                o[i] = __float_as_uint(f);
+              }
+              tmem_st_32x32b_x32(tbase + lane_base + 32 * c, o);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+          }
+          mbar_arrive(bar(B_OREADY + s));
+        }
+        if (!ok) break;
+        // ---- epilogue (line 20): out = O / (l * S16)
+        {
+          const uint32_t gl = gt - 1;
+          ok = mbar_wait(bar(B_PVDONE + (gl & 1)), (gl >> 1) & 1);
+          if (!ok) break;
+          ok = mbar_wait<true>(bar(B_FINFULL + (un & 1)), (un >> 1) & 1);
+          if (!ok) break;
+          tc_fence_after_sync();
+          float inv, lse;
+          {
+            uint32_t x, y;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(smem_base + kOffFin + ((un & 1) * 128 + r) * 8));
+            inv = __uint_as_float(x); lse = __uint_as_float(y);
+          }
+          const bool valid = r < u.nrows;
+          __nv_bfloat16* orow = prm.out + (static_cast<size_t>(u.b) * prm.R + u.r0 + r) * kDv;
+          float* prow = prm.part_o + (static_cast<size_t>(u.slot < 0 ? 0 : u.slot) * kRowBlock + r) * kDv;
+#pragma unroll 1
+          for (int c = 0; c < 16; ++c) {
+            uint32_t o[32];
+            tmem_ld_32x32b_x32(tbase + lane_base + 32 * c, o);
+            tmem_wait_ld();
+            if (valid) {
+              if (u.slot < 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  uint4 v;
+                  v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+                  v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+                  v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+                  v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+                  *reinterpret_cast<uint4*>(orow + 32 * c + 8 * i) = v;
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  float4 v = make_float4(__uint_as_float(o[4 * i + 0]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
+                                         __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv);
+                  *reinterpret_cast<float4*>(prow + 32 * c + 4 * i) = v;
+                }
+              }
+            }
+          }
+          if (valid) {
+            if (u.slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
+            else prm.part_lse[static_cast<size_t>(u.slot) * kRowBlock + r] = lse;
+          }
+          tc_fence_before_sync();
+        }
+        ++un;
+      }
+      if (!ok) report_timeout(prm.status);
+    } else if (wid == 4) {
+      // ---- TMA producer: V tiles (first 512 columns of the same cache rows)
+      if (lane == 0) {
+        uint32_t issued = 0;
+        while (ok && iter.next(u)) {
+          const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            const uint32_t stg = gt % kNumVStages, rnd = gt / kNumVStages;
+            ok = mbar_wait(bar(B_VEMPTY + stg), (rnd & 1) ^ 1);
+            if (!ok) break;
+            const int page = __ldg(bt + t);
+            mbar_arrive_expect_tx(bar(B_VFULL + stg), kVStageBytes);
+            const uint32_t dst = smem_base + kOffV + stg * kVStageBytes;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) tma_load_2d(dst + c * kBoxBytes, &kv_map, c * 64, page * kPage, bar(B_VFULL + stg));
+            ++issued;
+          }
+        }
+        if (!ok) {
+          report_timeout(prm.status);
+          for (uint32_t i = 0; i < kNumVStages && i < issued; ++i) {
+            const uint32_t n = issued - 1 - i;
+            mbar_wait(bar(B_VFULL + n % kNumVStages), (n / kNumVStages) & 1);
+          }
+        }
+      }
+    } else if (wid == 5) {
+      // ---- MMA issuer: O (+)= P~ V_t ; two N = 256 halves, four K = 16 steps each
+      if (lane == 0) {
+        constexpr uint32_t idesc = make_idesc_bf16(128, 256, false, true);
+        while (ok && iter.next(u)) {
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            const uint32_t stg = gt % kNumVStages, rnd = gt / kNumVStages;
+            const uint32_t s = gt & 1, k = gt >> 1;
+            ok = mbar_wait(bar(B_VFULL + stg), rnd & 1);
+            if (!ok) break;
+            ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
+            if (!ok) break;
+            ok = mbar_wait(bar(B_OREADY + s), k & 1);
+            if (!ok) break;
+            fence_proxy_async_all();
+            tc_fence_after_sync();
+            const uint32_t vbase = smem_base + kOffV + stg * kVStageBytes;
+            const uint32_t pbase = smem_base + kOffP + s * kPBytes;
+#pragma unroll
+            for (int nh = 0; nh < 2; ++nh) {
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t ad = make_smem_desc_sw128(pbase + kk * 32, 16, 1024);
+                const uint64_t bd = make_smem_desc_sw128(vbase + nh * 4 * kBoxBytes + kk * 2048, kBoxBytes, 1024);
+                mma_ss(tbase + nh * 256, ad, bd, idesc, (t > u.t0 || kk > 0) ? 1u : 0u);
+              }
+            }
+            mma_commit(bar(B_VEMPTY + stg));
+            mma_commit(bar(B_PVDONE + s));
+          }
+          if (!ok) break;
+        }
+        if (!ok) report_timeout(prm.status);
+      }
+    } else if (wid == 6) {
+      // ---- relay: tell the score CTA that a P buffer is free once its P V has completed
+      if (lane == 0) {
+        while (ok && iter.next(u)) {
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            const uint32_t s = gt & 1, k = gt >> 1;
+            ok = mbar_wait(bar(B_PVDONE + s), k & 1);
+            if (!ok) break;
+            mbar_arrive_cluster(peerA_bars + 8u * (A_PEMPTY + s));
+          }
+        }
+        if (!ok) report_timeout(prm.status);
+      }
+    }
+  }
+
+  // teardown: nobody may still be writing into a peer that has exited
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (wid == 5) tmem_dealloc(tbase, kTmemCols);
 }
+
+// ---------------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+template <int kMode, bool kGuard>
+cudaError_t launch_variant(const CUtensorMap& map, const DecodeParams& prm, cudaStream_t stream) {
+  auto kern = decode_tc_kernel<kMode, kGuard>;
+  cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  if (err != cudaSuccess) return err;
+  kern<<<2 * prm.P, kThreads, kSmemBytes, stream>>>(map, prm);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// Number of two-CTA clusters the schedule is cut into: one per SM pair.
+int decode_tc_parts(int sm_count) { return sm_count / 2 > 0 ? sm_count / 2 : 1; }
+
+cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* unsupported) {
+  *unsupported = 0;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) { *unsupported = 1; return cudaErrorNotSupported; }
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(kDqk), static_cast<cuuint64_t>(prm.num_blocks) * kPage};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(kDqk) * 2};
+  const cuuint32_t box[2] = {64, 64};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult cr = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(prm.kv), dims, strides,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  const int mode = prm.flags & 3;
+  const bool guard = !(prm.flags & 4);
+  if (mode == 0) return guard ? launch_variant<0, true>(map, prm, stream) : launch_variant<0, false>(map, prm, stream);
+  if (mode == 1) return guard ? launch_variant<1, true>(map, prm, stream) : launch_variant<1, false>(map, prm, stream);
+  return launch_variant<2, true>(map, prm, stream);
+}
+
+}  // namespace amla
