@@ -200,7 +200,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
 
           // lines 5-6: scale, mask, running max
           float tmax = -INFINITY;
-          if (t >= first_masked_tile || t < 0) {
+          if (t >= first_masked_tile) {
             const int jbase = t * kPage;
 #pragma unroll
             for (int i = 0; i < 64; ++i) {

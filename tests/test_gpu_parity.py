@@ -1,0 +1,139 @@
+"""GPU parity of the tensor-core decode path against the FP64 oracle, through the C-ABI, on identical
+seeded inputs.  Tolerances: max |err| <= 2e-2, relative L2 <= 5e-3 (bf16 output), |lse err| <= 1e-3."""
+import numpy as np
+import pytest
+
+from oracle import amla_sim as S
+from oracle import reference as R
+from paper_2509_25224_b200 import binding, synth
+from tests._gpu_util import check_full, check_sampled, run_gpu, to_device
+
+pytestmark = pytest.mark.gpu
+
+MODES = [binding.RESCALE_ALG2, binding.RESCALE_FOLD, binding.RESCALE_FMUL]
+
+
+def test_config1_tiny():
+    check_full(synth.config_tiny())
+
+
+@pytest.mark.parametrize("n", [1, 63, 64, 65, 128, 129, 1000])
+def test_single_sequence_lengths(n):
+    check_full(synth.make_workload("n", 1, 1, 128, [n], seed=200 + n))
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_ragged_batch_all_rescale_modes(mode):
+    # ragged lengths, an empty sequence, lengths shorter than Sq, Sq=2 causal rule, H=16 padding
+    w = synth.make_workload("r", 6, 2, 16, [300, 0, 1, 65, 1000, 2], seed=101)
+    check_full(w, mode)
+    w = synth.make_workload("r", 3, 1, 128, [700, 64, 129], seed=102)
+    check_full(w, mode)
+
+
+@pytest.mark.parametrize("Sq,H", [(1, 16), (1, 32), (1, 64), (2, 64), (2, 128), (3, 128), (4, 128), (1, 100), (3, 50)])
+def test_head_and_token_shapes(Sq, H):
+    w = synth.make_workload("s", 3, Sq, H, [200, 77, 513], seed=300 + 10 * Sq + H)
+    check_full(w)
+
+
+def test_all_sequences_empty():
+    w = synth.make_workload("e", 3, 2, 128, [0, 0, 0], seed=7)
+    out, lse, _ = run_gpu(w)
+    assert np.all(out == 0) and np.all(np.isneginf(lse))
+
+
+def test_many_short_sequences_more_items_than_parts():
+    rng = np.random.default_rng(9)
+    w = synth.make_workload("m", 200, 1, 128, rng.integers(0, 200, 200), seed=8)
+    check_full(w)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_staircase_rescale(mode):
+    check_full(synth.config_stress(B=2, N=4096), mode)
+
+
+def test_clamp_jump_and_falling_staircase():
+    n = 1024
+    w = synth.make_workload("j", 1, 1, 128, [n], seed=61)
+    synth.apply_logit_offsets(w, [np.where(np.arange(n) < 512, -30.0, 30.0)])
+    check_full(w)
+    w = synth.make_workload("f", 1, 1, 128, [n], seed=63)
+    synth.apply_logit_offsets(w, [synth.staircase_offsets(n)[::-1].copy()])
+    check_full(w)
+
+
+def test_exact_zero_v_columns_stay_zero():
+    w = synth.config_stress(B=1, N=2048)
+    w.kv[:, :, 100:110] = 0
+    out, lse, _ = run_gpu(w)
+    assert np.all(out[..., 100:110] == 0)
+    ro, rl = R.decode(w.q, w.kv, w.block_table, w.seqlens, w.scale)
+    from tests._gpu_util import compare
+    compare(out, lse, ro, rl, "zero columns")
+
+
+def test_large_magnitude_inputs():
+    # N(0, 3^2) inputs: logits spread ~ +-50, stresses the range handling of the recurrence.  The
+    # softmax is then nearly one-hot and |out| reaches ~12, where half a bf16 ulp of the output alone
+    # is 2^-5; the absolute tolerance is scaled with the value range (relative L2 and lse are not).
+    w = synth.make_workload("g", 2, 1, 128, [2000, 700], seed=12, sigma=3.0)
+    check_full(w, tol_abs=2e-2 * 4)
+    w = synth.make_workload("u", 2, 1, 128, [2000, 700], seed=13, dist="uniform", sigma=5.0)
+    check_full(w, tol_abs=2e-2 * 2)
+
+
+def test_rerun_is_bit_identical():
+    w = synth.make_workload("d", 4, 2, 128, [3000, 1000, 64, 4097], seed=33)
+    dev = to_device(w)
+    _, _, (o1, l1) = run_gpu(w, dev_inputs=dev)
+    _, _, (o2, l2) = run_gpu(w, dev_inputs=dev)
+    import torch
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
+
+
+def test_matches_algorithm2_simulator_closely():
+    # the CPU Algorithm-2 simulator uses the same readings; agreement should be far tighter than the
+    # oracle tolerance (both round P to bf16 and accumulate in fp32)
+    w = synth.config_stress(B=1, N=2048)
+    out, lse, _ = run_gpu(w)
+    kv = synth.bf16_bits_to_f32(synth.logical_kv_rows(w, 0))
+    q = synth.bf16_bits_to_f32(w.q[0, 0])
+    so, sl = S.amla(q, kv, kv[:, :512], w.scale, 64)
+    so = S.bf16_round(so)
+    assert np.abs(out[0, 0] - so).max() < 4e-3
+    assert np.abs(lse[0, 0] - sl).max() < 1e-4
+
+
+def test_error_codes_on_device():
+    import torch
+    w = synth.config_tiny()
+    q, kv, bt, sl = to_device(w)
+    out = torch.empty((1, 1, 16, 512), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((1, 1, 16), dtype=torch.float32, device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.AmlaError) as e:
+        binding.mla_decode(q, kv, bt, sl, w.scale, out, lse, small)
+    assert e.value.code == -3
+    with pytest.raises(binding.AmlaError) as e:
+        binding.mla_decode(q, kv, bt, sl, w.scale, out, lse, None, flags=3)
+    assert e.value.code == -1
+
+
+# ----------------------------------------------------------------- the five named configurations
+
+def test_config2_dsv3_sampled():
+    check_sampled(synth.config_dsv3(), 256)
+
+
+def test_config3_mtp_varlen_sampled():
+    check_sampled(synth.config_mtp(), 256)
+
+
+def test_config4_rescale_stress_sampled():
+    check_sampled(synth.config_stress(), 128)
+
+
+def test_config5_long_context_split_sampled():
+    check_sampled(synth.config_long(), 64)
