@@ -78,8 +78,8 @@ int amla_mla_decode_workspace_size(int B, int Sq, int H, int max_blocks_per_seq,
  *                need not be preserved or initialised; calls that overlap in time need distinct ones
  *   cuda_stream  a cudaStream_t (NULL = default stream)
  *
- * Supported: 1 <= Sq <= 8, 1 <= H <= 128 with Sq*H a multiple of 128 or smaller than 128 ... any Sq*H
- * up to 1024 rows; page size 64; sm_100 devices only (AMLA_ERR_UNSUPPORTED otherwise).
+ * Supported: 1 <= Sq <= 8, 1 <= H <= 128 (any Sq*H up to 1024 query rows per sequence; rows are
+ * processed in blocks of 128); page size 64; sm_100 devices only (AMLA_ERR_UNSUPPORTED otherwise).
  * Argument errors are reported before anything is launched.
  */
 int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_table,
@@ -100,6 +100,15 @@ int amla_check_status(const void* workspace, void* cuda_stream);
 
 /* Number of kernels the most recent amla_mla_decode[_ex] call on this thread launched. */
 int amla_last_launch_count(void);
+
+/* Measurement aid (the one piece of per-thread state in the library): when enabled, every decode call
+ * on this thread records CUDA events on its stream before and after each of its three launches
+ * (schedule, decode, combine).  The events are created on the first enable and live until exit. */
+int amla_profile_enable(int on);
+
+/* Waits for the last profiled call on this thread and writes the elapsed milliseconds of its three
+ * kernels (schedule, decode, combine) to ms3[0..2].  AMLA_ERR_INVALID_ARG if nothing was profiled. */
+int amla_profile_last_ms(float* ms3);
 
 /*
  * Host mirror of the device-side split-KV schedule (the plan is not in the paper; it exists because

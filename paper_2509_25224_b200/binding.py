@@ -23,7 +23,8 @@ FLAG_KERNEL_SIMT = 8
 
 EXPORTS = [
     "amla_status_string", "amla_mla_decode_workspace_size", "amla_mla_decode", "amla_mla_decode_ex",
-    "amla_check_status", "amla_last_launch_count", "amla_plan_host",
+    "amla_check_status", "amla_last_launch_count", "amla_plan_host", "amla_profile_enable",
+    "amla_profile_last_ms",
 ]
 
 _lib = None
@@ -59,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.amla_last_launch_count.restype = i32
         L.amla_plan_host.argtypes = [vp, i32, i32, i32, i32, vp, i32]
         L.amla_plan_host.restype = i32
+        L.amla_profile_enable.argtypes = [i32]
+        L.amla_profile_enable.restype = i32
+        L.amla_profile_last_ms.argtypes = [ctypes.POINTER(ctypes.c_float)]
+        L.amla_profile_last_ms.restype = i32
         _lib = L
     return _lib
 
@@ -102,6 +107,21 @@ def mla_decode_raw(q_ptr: int, kv_ptr: int, bt_ptr: int, sl_ptr: int, scale: flo
 
 def last_launch_count() -> int:
     return int(lib().amla_last_launch_count())
+
+
+def profile_enable(on: bool) -> None:
+    rc = lib().amla_profile_enable(1 if on else 0)
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_profile_enable")
+
+
+def profile_last_ms():
+    """(schedule_ms, decode_ms, combine_ms) of the last profiled call on this thread."""
+    ms = (ctypes.c_float * 3)()
+    rc = lib().amla_profile_last_ms(ms)
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_profile_last_ms")
+    return float(ms[0]), float(ms[1]), float(ms[2])
 
 
 def check_status(workspace, stream: int = 0) -> None:

@@ -52,6 +52,15 @@ int sm_count_of(int device, int* sms, int* cc_major) {
 
 thread_local int g_last_launches = 0;
 
+// Optional per-kernel timing (measurement aid): four events bracketing the three launches.
+thread_local bool g_profile = false;
+thread_local cudaEvent_t g_ev[4] = {nullptr, nullptr, nullptr, nullptr};
+thread_local bool g_ev_valid = false;
+
+void profile_mark(int i, cudaStream_t stream) {
+  if (g_profile && g_ev[i]) { cudaEventRecord(g_ev[i], stream); if (i == 3) g_ev_valid = true; }
+}
+
 }  // namespace
 }  // namespace amla
 
@@ -136,8 +145,10 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   prm.P = simt ? sms : decode_tc_parts(sms);
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  profile_mark(0, stream);
   if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
   ++g_last_launches;
+  profile_mark(1, stream);
   if (simt) {
     if (launch_decode_simt(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
   } else {
@@ -148,8 +159,10 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
     }
   }
   ++g_last_launches;
+  profile_mark(2, stream);
   if (launch_combine(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
   ++g_last_launches;
+  profile_mark(3, stream);
   return AMLA_OK;
 }
 
@@ -175,6 +188,27 @@ extern "C" int amla_check_status(const void* workspace, void* cuda_stream) {
 }
 
 extern "C" int amla_last_launch_count(void) { return g_last_launches; }
+
+extern "C" int amla_profile_enable(int on) {
+  if (on && !g_ev[0]) {
+    for (int i = 0; i < 4; ++i) {
+      if (cudaEventCreate(&g_ev[i]) != cudaSuccess) { cudaGetLastError(); g_ev[i] = nullptr; return AMLA_ERR_CUDA; }
+    }
+  }
+  g_profile = on != 0;
+  g_ev_valid = false;
+  return AMLA_OK;
+}
+
+extern "C" int amla_profile_last_ms(float* ms3) {
+  if (!ms3) return AMLA_ERR_INVALID_ARG;
+  if (!g_ev_valid) return AMLA_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(g_ev[3]) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  for (int i = 0; i < 3; ++i) {
+    if (cudaEventElapsedTime(&ms3[i], g_ev[i], g_ev[i + 1]) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  }
+  return AMLA_OK;
+}
 
 extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int num_parts, int32_t* units,
                               int max_units) {
