@@ -176,7 +176,10 @@ def run_gpu(args):
     out = torch.empty((B, Sq, H, 512), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((B, Sq, H), dtype=torch.float32, device=dev)
     ws = torch.empty(binding.workspace_size(B, Sq, H, w.max_blocks_per_seq, local), dtype=torch.uint8, device=dev)
-    flags = args.flags
+    flags = None if args.mode is None and args.tau is None else (
+        {"alg2": 0, "fold": 1, "fmul": 2}[args.mode or "alg2"] | binding.lazy(binding.DEFAULT_TAU if args.tau is None else args.tau)
+        | (binding.FLAG_UNGUARDED_ADD if args.unguarded else 0))
+    eff = binding.DEFAULT_FLAGS if flags is None else flags
 
     def step(i):
         q, kv, bt, sl = reps[i % nrep]
@@ -278,7 +281,7 @@ def run_gpu(args):
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(w), "l2": f"{nrep} input replicas rotated between steps "
-                       f"({nrep * kv_bytes / 1e6:.0f} MB of KV) > 126 MB L2", "rescale": ["alg2", "fold", "fmul"][flags & 3],
+                       f"({nrep * kv_bytes / 1e6:.0f} MB of KV) > 126 MB L2", "rescale": ["alg2", "fold", "fmul"][eff & 3] + f" tau={(eff >> 8) & 15}" + (" unguarded" if eff & 4 else ""),
                        "median_step_ms": statistics.median(per_step)},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": sess.h2d_bytes, "d2h_bytes_per_step": sess.d2h_bytes,
                     "steps": e2e_steps},
@@ -300,7 +303,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="dsv3", choices=list(synth.CONFIGS))
-    ap.add_argument("--flags", type=int, default=0, help="rescale variant: 0 alg2, 1 fold, 2 fmul (+4 unguarded)")
+    ap.add_argument("--mode", default=None, choices=["alg2", "fold", "fmul"], help="rescale variant (default: the library's)")
+    ap.add_argument("--tau", type=int, default=None, help="lazy-reference threshold in octaves, 0..15 (default: the library's)")
+    ap.add_argument("--unguarded", action="store_true", help="literal single integer add (measurement only)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

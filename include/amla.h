@@ -2,7 +2,7 @@
  * libamla -- paged MLA decode attention with exponent-add output rescaling (sm_100a).
  *
  * C ABI.  All pointers are borrowed; the library allocates no device memory and
- * keeps no state between calls.  Work is enqueued on the caller's stream with no
+ * keeps no state between calls beyond a per-device cache of device attributes.  Work is enqueued on the caller's stream with no
  * host synchronisation (sequence lengths are never read on the host).  Functions
  * return an amla_status; nothing throws, aborts or prints.
  *
@@ -40,6 +40,13 @@ typedef enum {
  *   AMLA_RESCALE_FMUL : Algorithm 1's FP32 multiply by exp(m_{i-1}-m_i) (the baseline the paper replaces).
  * AMLA_FLAG_UNGUARDED_ADD uses the literal single integer add of Algorithm 2 line 14 (corrupts
  * accumulators that are exactly 0.0 or below 2^-97; measurement only).
+ *
+ * AMLA_LAZY(tau), tau = 0..15 octaves: how far a tile's maximum may exceed the reference that P, l and
+ * the accumulator are expressed against before the reference is moved (and the accumulator rescaled).
+ * tau = 0 moves it with every new running maximum, which is Algorithm 2 to the letter.  With tau > 0
+ * the probabilities may reach 2^tau instead of 1 between moves -- harmless in bf16 P and FP32
+ * accumulators -- and rescales become rare; lines 6-12 of Algorithm 2 then run at the moves only.
+ * amla_mla_decode uses AMLA_RESCALE_ALG2 | AMLA_LAZY(AMLA_DEFAULT_TAU).
  */
 enum {
   AMLA_RESCALE_ALG2 = 0,
@@ -47,8 +54,12 @@ enum {
   AMLA_RESCALE_FMUL = 2,
   AMLA_RESCALE_MASK = 3,
   AMLA_FLAG_UNGUARDED_ADD = 4,
-  AMLA_FLAG_KERNEL_SIMT = 8     /* run the scalar bring-up kernel instead of the tensor-core kernel */
+  AMLA_FLAG_KERNEL_SIMT = 8,    /* run the scalar bring-up kernel instead of the tensor-core kernel */
+  AMLA_LAZY_SHIFT = 8,
+  AMLA_LAZY_MASK = 0xF00,
+  AMLA_DEFAULT_TAU = 8
 };
+#define AMLA_LAZY(tau) (((tau) & 0xF) << 8)
 
 /* Human-readable name of a status code (static storage). */
 const char* amla_status_string(int status);

@@ -20,6 +20,17 @@ RESCALE_FOLD = 1
 RESCALE_FMUL = 2
 FLAG_UNGUARDED_ADD = 4
 FLAG_KERNEL_SIMT = 8
+DEFAULT_TAU = 8
+
+
+def lazy(tau: int) -> int:
+    """Flag bits for a lazy-reference threshold of `tau` octaves (0 = Algorithm 2 to the letter)."""
+    if not 0 <= int(tau) <= 15:
+        raise ValueError("tau must be in 0..15")
+    return int(tau) << 8
+
+
+DEFAULT_FLAGS = RESCALE_ALG2 | lazy(DEFAULT_TAU)   # what amla_mla_decode (without _ex) uses
 
 EXPORTS = [
     "amla_status_string", "amla_mla_decode_workspace_size", "amla_mla_decode", "amla_mla_decode_ex",
@@ -97,10 +108,14 @@ def plan_host(seqlens, Sq: int, H: int, num_parts: int) -> np.ndarray:
 
 def mla_decode_raw(q_ptr: int, kv_ptr: int, bt_ptr: int, sl_ptr: int, scale: float, B: int, Sq: int, H: int,
                    num_blocks: int, max_blocks_per_seq: int, out_ptr: int, lse_ptr: int, ws_ptr: int,
-                   ws_bytes: int, stream: int = 0, flags: int = 0) -> None:
-    """amla_mla_decode_ex on raw device addresses."""
-    rc = lib().amla_mla_decode_ex(q_ptr, kv_ptr, bt_ptr, sl_ptr, float(scale), B, Sq, H, num_blocks,
-                                  max_blocks_per_seq, out_ptr, lse_ptr, ws_ptr, ws_bytes, stream, flags)
+                   ws_bytes: int, stream: int = 0, flags: int | None = None) -> None:
+    """amla_mla_decode (flags None) or amla_mla_decode_ex on raw device addresses."""
+    if flags is None:
+        rc = lib().amla_mla_decode(q_ptr, kv_ptr, bt_ptr, sl_ptr, float(scale), B, Sq, H, num_blocks,
+                                   max_blocks_per_seq, out_ptr, lse_ptr, ws_ptr, ws_bytes, stream)
+    else:
+        rc = lib().amla_mla_decode_ex(q_ptr, kv_ptr, bt_ptr, sl_ptr, float(scale), B, Sq, H, num_blocks,
+                                      max_blocks_per_seq, out_ptr, lse_ptr, ws_ptr, ws_bytes, stream, int(flags))
     if rc != AMLA_OK:
         raise AmlaError(rc, "amla_mla_decode")
 
@@ -131,7 +146,7 @@ def check_status(workspace, stream: int = 0) -> None:
 
 
 def mla_decode(q, kv_cache, block_table, seqlens, softmax_scale: float, out=None, lse=None, workspace=None,
-               flags: int = 0):
+               flags: int | None = None):
     """Device tensors in, device tensors out (torch is the allocator and stream provider).
 
     q bf16 [B,Sq,H,576], kv_cache bf16 [num_blocks,64,576], block_table int32 [B,max_blocks],
@@ -204,7 +219,7 @@ class HostSession:
     def d2h_bytes(self):
         return sum(x.numel() * x.element_size() for x in (self.h_out, self.h_lse))
 
-    def run(self, scale, flags=0, sync=True):
+    def run(self, scale, flags=None, sync=True):
         self.d_q.copy_(self.h_q, non_blocking=True)
         self.d_kv.copy_(self.h_kv, non_blocking=True)
         self.d_bt.copy_(self.h_bt, non_blocking=True)

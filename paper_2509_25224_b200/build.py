@@ -28,6 +28,15 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def build_trace() -> str:
+    """Developer aid: libamla_trace.so, the same sources with -DAMLA_TRACE (per-role cycle stamps)."""
+    out = os.path.join(_HERE, "libamla_trace.so")
+    nvcc = os.environ.get("NVCC", "nvcc")
+    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")] + ["-DAMLA_TRACE"]
+    subprocess.check_call([nvcc] + flags + sources() + ["-o", out])
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
@@ -43,4 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
+    if "--trace" in sys.argv:
+        print(build_trace())
+        sys.exit(0)
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

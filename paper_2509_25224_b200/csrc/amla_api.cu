@@ -1,5 +1,6 @@
 // C-ABI entry points of libamla: argument validation, workspace carving and the three launches
 // (schedule prefix, decode, combine) on the caller's stream.
+#include <atomic>
 #include <cstring>
 
 #include "../../include/amla.h"
@@ -42,15 +43,33 @@ int check_shape(int B, int Sq, int H, int max_blocks_per_seq) {
   return AMLA_OK;
 }
 
+// SM count and compute capability per device, queried once (the attributes never change).
+constexpr int kMaxDevices = 64;
+struct DeviceInfo { std::atomic<int> ready{0}; int sms = 0; int cc_major = 0; };
+DeviceInfo g_devices[kMaxDevices];
+
 int sm_count_of(int device, int* sms, int* cc_major) {
-  cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-  *sms = prop.multiProcessorCount;
-  *cc_major = prop.major;
+  if (device < 0 || device >= kMaxDevices) return AMLA_ERR_INVALID_ARG;
+  DeviceInfo& d = g_devices[device];
+  if (!d.ready.load(std::memory_order_acquire)) {
+    int s = 0, c = 0;
+    if (cudaDeviceGetAttribute(&s, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) {
+      cudaGetLastError();
+      return AMLA_ERR_CUDA;
+    }
+    d.sms = s; d.cc_major = c;
+    d.ready.store(1, std::memory_order_release);
+  }
+  *sms = d.sms;
+  *cc_major = d.cc_major;
   return AMLA_OK;
 }
 
 thread_local int g_last_launches = 0;
+#ifdef AMLA_TRACE
+thread_local unsigned long long* g_trace = nullptr;
+#endif
 
 // Optional per-kernel timing (measurement aid): four events bracketing the three launches.
 thread_local bool g_profile = false;
@@ -141,6 +160,10 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   prm.num_blocks = num_blocks;
   prm.max_blocks_per_seq = max_blocks_per_seq;
   prm.flags = flags;
+#ifdef AMLA_TRACE
+  prm.trace = g_trace;
+#endif
+  prm.tau = static_cast<float>((flags & AMLA_LAZY_MASK) >> AMLA_LAZY_SHIFT);
   const bool simt = (flags & AMLA_FLAG_KERNEL_SIMT) != 0;
   prm.P = simt ? sms : decode_tc_parts(sms);
 
@@ -172,7 +195,7 @@ extern "C" int amla_mla_decode(const void* q, const void* kv_cache, const int32_
                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return amla_mla_decode_ex(q, kv_cache, block_table, seqlens, softmax_scale, B, Sq, H, num_blocks,
                             max_blocks_per_seq, out, lse, workspace, workspace_bytes, cuda_stream,
-                            AMLA_RESCALE_ALG2);
+                            AMLA_RESCALE_ALG2 | AMLA_LAZY(AMLA_DEFAULT_TAU));
 }
 
 extern "C" int amla_check_status(const void* workspace, void* cuda_stream) {
@@ -255,3 +278,12 @@ extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int 
   delete[] prefix;
   return overflow ? AMLA_ERR_WORKSPACE : n_units;
 }
+
+#ifdef AMLA_TRACE
+// Trace builds only (not part of the public header): device buffer of
+// parts * kTraceEvents * kTraceTiles 64-bit stamps that later calls on this thread fill.
+extern "C" int amla_debug_set_trace(void* device_buffer) {
+  g_trace = static_cast<unsigned long long*>(device_buffer);
+  return AMLA_OK;
+}
+#endif

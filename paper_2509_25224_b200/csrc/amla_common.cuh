@@ -31,6 +31,7 @@ struct DecodeParams {
   float* part_o;                 // [2 * P, 128, 512] fp32 normalised partial outputs
   float* part_lse;               // [2 * P, 128]      partial lse (natural log)
   float scale_log2;              // softmax_scale * log2(e)
+  float tau;                     // lazy-reference threshold in octaves (0 = move the reference with every new maximum)
   int B, Sq, H;
   int R;                         // Sq * H query rows per sequence
   int nrb;                       // row blocks per sequence = ceil(R / 128)
@@ -38,7 +39,23 @@ struct DecodeParams {
   int num_blocks, max_blocks_per_seq;
   int P;                         // parts the linear tile range is cut into
   int flags;
+  unsigned long long* trace;     // timeline buffer of a -DAMLA_TRACE build, else unused (nullptr)
 };
+
+// Optional per-role timeline (compiled in with -DAMLA_TRACE only): every stamp is the SM's cycle
+// counter, stored at trace[(part * kTraceEvents + event) * kTraceTiles + index].
+constexpr int kTraceEvents = 24;
+constexpr int kTraceTiles = 96;
+#ifdef AMLA_TRACE
+#define AMLA_STAMP(prm, part, ev, idx)                                                                      \
+  do {                                                                                                      \
+    if ((prm).trace && static_cast<unsigned>(idx) < static_cast<unsigned>(amla::kTraceTiles))                \
+      (prm).trace[(static_cast<size_t>(part) * amla::kTraceEvents + (ev)) * amla::kTraceTiles + (idx)] =     \
+          static_cast<unsigned long long>(clock64());                                                       \
+  } while (0)
+#else
+#define AMLA_STAMP(prm, part, ev, idx) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // Split-KV schedule.  Items (sequence b, row block rb) in order it = b * nrb + rb own
@@ -122,18 +139,23 @@ __device__ __forceinline__ float bf16_round(float x) {
 // ---------------------------------------------------------------------------------------------
 // Per-row running state and the scalar part of one tile step, in the base-2 domain:
 // a_j = s_j * log2(e), so exp(s_j - m) = 2^(a_j - m2) and n_i = round(-m_i / ln 2) = round(-m2).
+//
+// The reference m2 that P, l and O are expressed against is the running maximum of Algorithm 2 when
+// tau == 0.  With tau > 0 it is moved only when a tile's maximum exceeds it by more than tau octaves
+// (then to that maximum); in between P may reach 2^tau instead of 1, which bf16 P and the FP32
+// accumulators hold without loss, and the accumulator needs no rescale.  Lines 6-12 of Algorithm 2
+// are evaluated at the moves, with the stale reference in the place of m_{i-1}.
 // ---------------------------------------------------------------------------------------------
 struct RowState {
-  float m2;      // running max of a_j (-inf before the first visible key)
-  float l;       // running row sum of P (unscaled FP32, Algorithm 2 line 6)
-  float n;       // n_i of the last tile with a visible key
-  float c;       // c_i of that tile (Appendix A: r_i / r'_i = S16 / S32)
-  float s_out;   // scale folded into P for that tile (S16, S32 or 1 depending on the mode)
-  int started;   // the row's accumulator has received a P V product
+  float m2;      // reference of a_j (-inf before the first visible key)
+  float l;       // running row sum of P against that reference (unscaled FP32, Algorithm 2 line 6)
+  float n;       // n_i of the last move
+  float c;       // c_i of the last move (Appendix A: r_i / r'_i = S16 / S32)
+  float s_out;   // scale folded into P since the last move (S16, S32 or 1 depending on the mode)
 };
 
 __device__ __forceinline__ void row_state_init(RowState& st) {
-  st.m2 = -INFINITY; st.l = 0.f; st.n = 0.f; st.c = 1.f; st.s_out = 1.f; st.started = 0;
+  st.m2 = -INFINITY; st.l = 0.f; st.n = 0.f; st.c = 1.f; st.s_out = 1.f;
 }
 
 // Result of the scalar step for one row and one tile.
@@ -146,46 +168,45 @@ struct RowStep {
 
 // mode: 0 = Algorithm 2, 1 = exact fold (Eq. 3), 2 = FP32 multiply (Algorithm 1).
 template <int kMode>
-__device__ __forceinline__ RowStep row_step(RowState& st, float tile_max2) {
+__device__ __forceinline__ RowStep row_step(RowState& st, float tile_max2, float tau) {
   RowStep r;
   const float m_old = st.m2;
-  const float m_new = fmaxf(m_old, tile_max2);
-  if (m_new == -INFINITY) {        // nothing visible so far: P will be all zeros
-    r.m2_sub = 0.f; r.p_scale = 1.f; r.l_up = 1.f; r.n_bits = 0;
+  r.n_bits = 0;
+  r.l_up = 1.f;
+  if (!(tile_max2 > m_old + tau)) {   // reference stays (also: nothing visible in this tile)
+    r.m2_sub = (m_old == -INFINITY) ? 0.f : m_old;
+    r.p_scale = st.s_out;
     return r;
   }
+  const float m_new = tile_max2;     // > m_old
+  const bool started = m_old != -INFINITY;
   r.m2_sub = m_new;
-  r.l_up = (m_old == -INFINITY) ? 0.f : ex2_approx(m_old - m_new);
-  r.n_bits = 0;
+  r.l_up = started ? ex2_approx(m_old - m_new) : 0.f;
   if (kMode == 2) {
     r.p_scale = 1.f;
     st.s_out = 1.f;
   } else {
     const float n_i = rintf(-m_new);                       // Alg. 2 line 6
     const float s32 = ex2_approx(n_i + m_new);             // line 7: 1/r_i in [1/sqrt2, sqrt2]
+    const int dn = static_cast<int>(fmaxf(n_i - st.n, -30.f));   // line 11
     if (kMode == 0) {
       const float s16 = bf16_round(s32);                   // line 8
       const float c_i = __fdividef(s16, s32);              // Appendix A: c_i = r_i / r'_i
-      if (st.started && m_new != m_old) {
+      if (started) {
         const float eps = 1.5f * (__fdividef(c_i, st.c) - 1.f);           // line 9
-        const int dn = static_cast<int>(fmaxf(n_i - st.n, -30.f));        // line 11
         r.n_bits = dn * (1 << 23) + __float2int_rn((eps + 1e-6f) * 8388608.f);   // line 12
       }
       st.c = c_i;
       r.p_scale = s16;                                     // line 10
       st.s_out = s16;
     } else {
-      if (st.started && n_i != st.n) {
-        const int dn = static_cast<int>(fmaxf(n_i - st.n, -30.f));
-        r.n_bits = dn * (1 << 23);
-      }
+      if (started) r.n_bits = dn * (1 << 23);              // 0 when n_i did not change
       r.p_scale = s32;
       st.s_out = s32;
     }
     st.n = n_i;
   }
   st.m2 = m_new;
-  st.started = 1;
   return r;
 }
 

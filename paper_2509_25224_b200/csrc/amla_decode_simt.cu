@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
 #pragma unroll
           for (int o = 16; o; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
           // V1: scalar recurrence + probabilities
-          const RowStep sp = row_step<kMode>(st[rr], tmax);
+          const RowStep sp = row_step<kMode>(st[rr], tmax, prm.tau);
           const float p0 = ex2_approx(a0 - sp.m2_sub), p1 = ex2_approx(a1 - sp.m2_sub);
           float rs = p0 + p1;
 #pragma unroll

@@ -18,6 +18,8 @@
 // so the integer add is a TMEM load/add/store rather than an atomic in global memory.
 //
 // All waits are bounded; on expiry the kernel records kStatusTimeout and unwinds.
+#include <atomic>
+
 #include "amla_common.cuh"
 #include "amla_sm100.cuh"
 
@@ -139,6 +141,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
   tc_fence_after_sync();
   uint32_t tbase;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tbase) : "r"(tmem_slot));
+  if (tid == 0) AMLA_STAMP(prm, part, is_score ? 0 : 1, 0);
 
   bool ok = true;
   UnitIter iter(prm, part);
@@ -157,6 +160,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
         ok = mbar_wait(bar(A_QFREE), (un & 1) ^ 1);
         if (!ok) break;
         tc_fence_after_sync();
+        if (tid == 0) AMLA_STAMP(prm, part, 10, un);
         {
           const bool valid = r < u.nrows;
           const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDqk);
@@ -174,18 +178,21 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
         }
         tc_fence_before_sync();
         mbar_arrive(bar(A_QREADY));
+        if (tid == 0) AMLA_STAMP(prm, part, 11, un);
 
         RowState st;
         row_state_init(st);
         const int tok = (u.r0 + r) / prm.H;
         const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);   // keys 0..visible-1 are seen by this row
-        const int first_masked_tile = (u.n_b - prm.Sq + 1) / kPage;  // tiles from here on may hold hidden keys
+        const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // tiles from here on may hold hidden keys
+        const bool scale_nonneg = prm.scale_log2 >= 0.f;
 
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
           const uint32_t s = gt & 1, k = gt >> 1;
           ok = mbar_wait(bar(A_SFULL + s), k & 1);
           if (!ok) break;
           tc_fence_after_sync();
+          if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
           uint32_t a[64];
           {
             uint32_t lo[32], hi[32];
@@ -197,42 +204,57 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
           }
           tc_fence_before_sync();
           mbar_arrive(bar(A_SEMPTY + s));
+          if (tid == 0) AMLA_STAMP(prm, part, 6, gt);
 
-          // lines 5-6: scale, mask, running max
-          float tmax = -INFINITY;
+          // lines 5-6: mask, running max (taken on the raw scores; the scale is folded into the FMA below)
+          const int nvis = visible - t * kPage;            // keys of this tile the row sees (may be <= 0 or >= 64)
           if (t >= first_masked_tile) {
-            const int jbase = t * kPage;
+            const uint32_t fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
 #pragma unroll
-            for (int i = 0; i < 64; ++i) {
-              float v = __uint_as_float(a[i]) * prm.scale_log2;
-              v = (jbase + i < visible) ? v : -INFINITY;
-              a[i] = __float_as_uint(v);
-              tmax = fmaxf(tmax, v);
+            for (int i = 0; i < 64; ++i) a[i] = (i < nvis) ? a[i] : fill;
+          }
+          float ext;
+          if (scale_nonneg) {
+            ext = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 64; i += 2) ext = fmax3(ext, __uint_as_float(a[i]), __uint_as_float(a[i + 1]));
+          } else {
+            ext = INFINITY;
+#pragma unroll
+            for (int i = 0; i < 64; i += 2) ext = fminf(ext, fminf(__uint_as_float(a[i]), __uint_as_float(a[i + 1])));
+          }
+          const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
+          const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
+          // lines 6, 10: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
+          float rs0 = 0.f, rs1 = 0.f;
+          uint32_t pk[32];
+          const float nsub = -sp.m2_sub;
+          if (t >= first_masked_tile) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
+              float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
+              p0 = (2 * i < nvis) ? p0 : 0.f;
+              p1 = (2 * i + 1 < nvis) ? p1 : 0.f;
+              rs0 += p0; rs1 += p1;
+              pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
             }
           } else {
 #pragma unroll
-            for (int i = 0; i < 64; ++i) {
-              const float v = __uint_as_float(a[i]) * prm.scale_log2;
-              a[i] = __float_as_uint(v);
-              tmax = fmaxf(tmax, v);
+            for (int i = 0; i < 32; ++i) {
+              const float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
+              const float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
+              rs0 += p0; rs1 += p1;
+              pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
             }
           }
-          const RowStep sp = row_step<kMode>(st, tmax);
-          // lines 6, 10: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
-          float rs = 0.f;
-          uint32_t pk[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float p0 = ex2_approx(__uint_as_float(a[2 * i]) - sp.m2_sub);
-            const float p1 = ex2_approx(__uint_as_float(a[2 * i + 1]) - sp.m2_sub);
-            rs += p0 + p1;
-            pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
-          }
-          st.l = st.l * sp.l_up + rs;
+          st.l = st.l * sp.l_up + (rs0 + rs1);
 
           // hand P~ and N to the value CTA
+          if (tid == 0) AMLA_STAMP(prm, part, 7, gt);
           ok = mbar_wait(bar(A_PEMPTY + s), (k & 1) ^ 1);
           if (!ok) break;
+          if (tid == 0) AMLA_STAMP(prm, part, 8, gt);
           const uint32_t pdst = peerB_base + kOffP + s * kPBytes;
 #pragma unroll
           for (int c = 0; c < 8; ++c)
@@ -241,6 +263,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
           st_cluster_b32(peerB_base + kOffN + (s * 128 + r) * 4, nword);
           fence_proxy_async_all();
           mbar_arrive_cluster(peerB_bars + 8u * (B_PFULL + s));
+          if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
         }
         if (!ok) break;
         // line 20 scalars: 1 / (l * S16) and lse = m + ln l
@@ -266,6 +289,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             const uint32_t stg = gt % kNumKStages, rnd = gt / kNumKStages;
             ok = mbar_wait(bar(A_KEMPTY + stg), (rnd & 1) ^ 1);
             if (!ok) break;
+            AMLA_STAMP(prm, part, 2, gt);
             const int page = __ldg(bt + t);
             mbar_arrive_expect_tx(bar(A_KFULL + stg), kKStageBytes);
             const uint32_t dst = smem_base + kOffK + stg * kKStageBytes;
@@ -299,6 +323,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             ok = mbar_wait(bar(A_SEMPTY + s), (k & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
+            AMLA_STAMP(prm, part, 3, gt);
             const uint32_t kbase = smem_base + kOffK + stg * kKStageBytes;
             const uint32_t d = tbase + kSCol + 64 * s;
 #pragma unroll
@@ -308,6 +333,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             }
             mma_commit(bar(A_KEMPTY + stg));
             mma_commit(bar(A_SFULL + s));
+            AMLA_STAMP(prm, part, 4, gt);
           }
           if (!ok) break;
           mma_commit(bar(A_QFREE));
@@ -327,6 +353,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
           const uint32_t s = gt & 1, k = gt >> 1;
           ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
           if (!ok) break;
+          if (tid == 0) AMLA_STAMP(prm, part, 13, gt);
           uint32_t nword;
           asm volatile("ld.shared.b32 %0, [%1];" : "=r"(nword) : "r"(smem_base + kOffN + (s * 128 + r) * 4));
           const bool mine = (kMode == 2) ? (__uint_as_float(nword) != 1.f) : (nword != 0u);
@@ -336,11 +363,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             ok = mbar_wait(bar(B_PVDONE + (gp & 1)), (gp >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
-#pragma unroll 1
-            for (int c = 0; c < 16; ++c) {
-              uint32_t o[32];
-              tmem_ld_32x32b_x32(tbase + lane_base + 32 * c, o);
-              tmem_wait_ld();
+            // two 32-column chunks in flight: the load of one overlaps the arithmetic of the other
+            auto apply = [&](uint32_t (&o)[32]) {
 #pragma unroll
               for (int i = 0; i < 32; ++i) {
                 float f = __uint_as_float(o[i]);
@@ -348,12 +372,26 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
                 else f = kGuard ? exponent_add_guarded(f, static_cast<int>(nword)) : exponent_add_raw(f, static_cast<int>(nword));
                 o[i] = __float_as_uint(f);
               }
-              tmem_st_32x32b_x32(tbase + lane_base + 32 * c, o);
+            };
+            uint32_t o0[32], o1[32];
+            const uint32_t obase = tbase + lane_base;
+            tmem_ld_32x32b_x32(obase, o0);
+#pragma unroll 1
+            for (int c = 0; c < 16; c += 2) {
+              tmem_wait_ld();
+              tmem_ld_32x32b_x32(obase + 32 * (c + 1), o1);
+              apply(o0);
+              tmem_st_32x32b_x32(obase + 32 * c, o0);
+              tmem_wait_ld();
+              if (c + 2 < 16) tmem_ld_32x32b_x32(obase + 32 * (c + 2), o0);
+              apply(o1);
+              tmem_st_32x32b_x32(obase + 32 * (c + 1), o1);
             }
             tmem_wait_st();
             tc_fence_before_sync();
           }
           mbar_arrive(bar(B_OREADY + s));
+          if (tid == 0) AMLA_STAMP(prm, part, 14, gt);
         }
         if (!ok) break;
         // ---- epilogue (line 20): out = O / (l * S16)
@@ -364,6 +402,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
           ok = mbar_wait<true>(bar(B_FINFULL + (un & 1)), (un >> 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
+          if (tid == 0) AMLA_STAMP(prm, part, 18, un);
           float inv, lse;
           {
             uint32_t x, y;
@@ -404,6 +443,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             else prm.part_lse[static_cast<size_t>(u.slot) * kRowBlock + r] = lse;
           }
           tc_fence_before_sync();
+          if (tid == 0) AMLA_STAMP(prm, part, 19, un);
         }
         ++un;
       }
@@ -418,6 +458,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             const uint32_t stg = gt % kNumVStages, rnd = gt / kNumVStages;
             ok = mbar_wait(bar(B_VEMPTY + stg), (rnd & 1) ^ 1);
             if (!ok) break;
+            AMLA_STAMP(prm, part, 12, gt);
             const int page = __ldg(bt + t);
             mbar_arrive_expect_tx(bar(B_VFULL + stg), kVStageBytes);
             const uint32_t dst = smem_base + kOffV + stg * kVStageBytes;
@@ -450,6 +491,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             if (!ok) break;
             fence_proxy_async_all();
             tc_fence_after_sync();
+            AMLA_STAMP(prm, part, 15, gt);
             const uint32_t vbase = smem_base + kOffV + stg * kVStageBytes;
             const uint32_t pbase = smem_base + kOffP + s * kPBytes;
 #pragma unroll
@@ -463,6 +505,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             }
             mma_commit(bar(B_VEMPTY + stg));
             mma_commit(bar(B_PVDONE + s));
+            AMLA_STAMP(prm, part, 16, gt);
           }
           if (!ok) break;
         }
@@ -476,6 +519,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
             const uint32_t s = gt & 1, k = gt >> 1;
             ok = mbar_wait(bar(B_PVDONE + s), k & 1);
             if (!ok) break;
+            AMLA_STAMP(prm, part, 17, gt);
             mbar_arrive_cluster(peerA_bars + 8u * (A_PEMPTY + s));
           }
         }
@@ -516,8 +560,17 @@ EncodeTiledFn get_encode_fn() {
 template <int kMode, bool kGuard>
 cudaError_t launch_variant(const CUtensorMap& map, const DecodeParams& prm, cudaStream_t stream) {
   auto kern = decode_tc_kernel<kMode, kGuard>;
-  cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  // the opt-in to large dynamic shared memory is per device and per kernel; do it once each
+  static std::atomic<uint64_t> done{0};
+  int device = 0;
+  cudaError_t err = cudaGetDevice(&device);
   if (err != cudaSuccess) return err;
+  const uint64_t bit = 1ull << (device & 63);
+  if (!(done.load(std::memory_order_acquire) & bit)) {
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+    if (err != cudaSuccess) return err;
+    done.fetch_or(bit, std::memory_order_release);
+  }
   kern<<<2 * prm.P, kThreads, kSmemBytes, stream>>>(map, prm);
   return cudaGetLastError();
 }

@@ -21,7 +21,7 @@ def to_device(w):
     return q, kv, bt, sl
 
 
-def run_gpu(w, flags=0, poison=True, dev_inputs=None):
+def run_gpu(w, flags=None, poison=True, dev_inputs=None):
     """Returns (out float64 [B,Sq,H,512], lse float64 [B,Sq,H]) computed by the CUDA path."""
     import torch
     q, kv, bt, sl = dev_inputs if dev_inputs is not None else to_device(w)
@@ -53,13 +53,13 @@ def compare(out, lse, ref_out, ref_lse, what="", tol_abs=TOL_ABS):
     return float(err.max()), float(rel)
 
 
-def check_full(w, flags=0, what="", tol_abs=TOL_ABS):
+def check_full(w, flags=None, what="", tol_abs=TOL_ABS):
     out, lse, _ = run_gpu(w, flags)
     ro, rl = R.decode(w.q, w.kv, w.block_table, w.seqlens, w.scale)
     return compare(out, lse, ro, rl, what or w.name, tol_abs)
 
 
-def check_sampled(w, n_rows=192, flags=0, seed=0, what="", dev_inputs=None):
+def check_sampled(w, n_rows=192, flags=None, seed=0, what="", dev_inputs=None):
     """Full-size workloads: compare a seeded sample of (b,t,h) rows, plus finiteness everywhere."""
     out, lse, _ = run_gpu(w, flags, dev_inputs=dev_inputs)
     assert np.isfinite(out).all()

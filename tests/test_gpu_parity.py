@@ -10,7 +10,10 @@ from tests._gpu_util import check_full, check_sampled, run_gpu, to_device
 
 pytestmark = pytest.mark.gpu
 
-MODES = [binding.RESCALE_ALG2, binding.RESCALE_FOLD, binding.RESCALE_FMUL]
+# every rescale variant, with the reference moved at every new maximum (tau = 0: Algorithm 2 to the
+# letter) and lazily (tau = 8 octaves, the default of amla_mla_decode)
+MODES = [m | binding.lazy(tau) for m in (binding.RESCALE_ALG2, binding.RESCALE_FOLD, binding.RESCALE_FMUL)
+         for tau in (0, 8)] + [binding.RESCALE_ALG2 | binding.lazy(2)]
 
 
 def test_config1_tiny():
@@ -54,14 +57,15 @@ def test_staircase_rescale(mode):
     check_full(synth.config_stress(B=2, N=4096), mode)
 
 
-def test_clamp_jump_and_falling_staircase():
+@pytest.mark.parametrize("flags", [None, binding.RESCALE_ALG2, binding.RESCALE_FOLD | binding.lazy(4)])
+def test_clamp_jump_and_falling_staircase(flags):
     n = 1024
     w = synth.make_workload("j", 1, 1, 128, [n], seed=61)
     synth.apply_logit_offsets(w, [np.where(np.arange(n) < 512, -30.0, 30.0)])
-    check_full(w)
+    check_full(w, flags)
     w = synth.make_workload("f", 1, 1, 128, [n], seed=63)
     synth.apply_logit_offsets(w, [synth.staircase_offsets(n)[::-1].copy()])
-    check_full(w)
+    check_full(w, flags)
 
 
 def test_exact_zero_v_columns_stay_zero():
@@ -97,7 +101,7 @@ def test_matches_algorithm2_simulator_closely():
     # the CPU Algorithm-2 simulator uses the same readings; agreement should be far tighter than the
     # oracle tolerance (both round P to bf16 and accumulate in fp32)
     w = synth.config_stress(B=1, N=2048)
-    out, lse, _ = run_gpu(w)
+    out, lse, _ = run_gpu(w, binding.RESCALE_ALG2)          # tau = 0, as the simulator
     kv = synth.bf16_bits_to_f32(synth.logical_kv_rows(w, 0))
     q = synth.bf16_bits_to_f32(w.q[0, 0])
     so, sl = S.amla(q, kv, kv[:, :512], w.scale, 64)
@@ -132,7 +136,10 @@ def test_config3_mtp_varlen_sampled():
 
 
 def test_config4_rescale_stress_sampled():
-    check_sampled(synth.config_stress(), 128)
+    w = synth.config_stress()
+    dev = to_device(w)
+    check_sampled(w, 128, dev_inputs=dev)
+    check_sampled(w, 64, flags=binding.RESCALE_ALG2, dev_inputs=dev)   # tau = 0
 
 
 def test_config5_long_context_split_sampled():
