@@ -1,21 +1,24 @@
 // Tensor-core MLA decode kernel for sm_100a.
 //
-// A cluster of two CTAs works on one 128-row block of query rows and a range of 64-key tiles:
+// A cluster of two CTAs works on one 128-row block of query rows and a range of 64-key cache pages:
 //
-//   score CTA (cluster rank 0)   Q (128 x 576 bf16) resident in tensor memory as the A operand;
-//       K tiles streamed by TMA; S = Q K^T by tcgen05.mma into a double-buffered TMEM tile; the
-//       softmax warpgroup runs Algorithm 2's per-row recurrence (lines 5-12) and writes the bf16
-//       probabilities P~ = bf16(P * S16) and the per-row integer N into the value CTA's shared
-//       memory (distributed shared memory).
+//   score CTA (cluster rank 0)   the 512 latent columns of Q (128 x 512 bf16) are resident in tensor
+//       memory as the A operand, the 64 RoPE columns in shared memory.  K arrives by TMA in slots of
+//       128 keys x 64 columns (two pages stacked), nine slots per score tile, through an 11-slot
+//       ring; S = Q K^T (128 x 128, FP32) by tcgen05.mma into a double-buffered TMEM tile.  The
+//       softmax warpgroup runs Algorithm 2's per-row recurrence (lines 5-12) once per score tile,
+//       writes the bf16 probabilities P~ = bf16(P * S16) of each 64-key half plus the per-row integer
+//       N into a local staging buffer, and a bulk shared-to-shared copy moves it into the value CTA.
 //   value CTA (cluster rank 1)   the whole FP32 accumulator O (128 x 512) lives in its tensor memory;
-//       V tiles (first 512 columns of the same cache rows) streamed by TMA; a correction warpgroup
-//       applies N to the bit patterns of O (lines 13-16; Lemma 3.1) for rows whose maximum moved,
-//       then O += P~ V by tcgen05.mma (lines 17-18); the epilogue divides by l * S16 (line 20).
+//       V (first 512 columns of the same cache rows) arrives by TMA in slots of 64 keys x 256
+//       columns through a 5-slot ring; a correction warpgroup applies N to the bit patterns of O
+//       (lines 13-16; Lemma 3.1) for rows whose reference moved, then O += P~ V by tcgen05.mma
+//       (lines 17-18); the epilogue divides by l * S16 (line 20).
 //
 // This is the counterpart of the paper's split between matrix and vector units (Section 3.3) with
-// its [C1, C2, V1] steady-state order (Section 4.1): QK^T of tile i+1 is issued before P V of tile i
-// finishes, and the softmax of tile i+1 overlaps both.  What differs: O never leaves tensor memory,
-// so the integer add is a TMEM load/add/store rather than an atomic in global memory.
+// its [C1, C2, V1] steady-state order (Section 4.1): QK^T of the next tile is issued before P V of
+// this one finishes, and the softmax overlaps both.  What differs: O never leaves tensor memory, so
+// the integer add is a TMEM load/add/store rather than an atomic in global memory.
 //
 // All waits are bounded; on expiry the kernel records kStatusTimeout and unwinds.
 #include <atomic>
@@ -29,38 +32,44 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kThreads = 224;            // warps 0-3: softmax / correction, 4: TMA, 5: MMA + TMEM alloc, 6: relay
-constexpr int kNumKStages = 3;
-constexpr int kNumVStages = 2;
+constexpr int kThreads = 224;            // warps 0-3: softmax / correction, 4: TMA, 5: MMA + TMEM alloc, 6: copy / relay
 constexpr uint32_t kBoxBytes = 64 * 64 * 2;             // one 64-key x 64-column TMA box
-constexpr uint32_t kKStageBytes = 9 * kBoxBytes;        // 73728
-constexpr uint32_t kVStageBytes = 8 * kBoxBytes;        // 65536
-constexpr uint32_t kPBytes = 128 * 64 * 2;              // 16384
+constexpr uint32_t kPBytes = 128 * 64 * 2;              // P~ of one 64-key half: 128 rows x 128 B
+constexpr uint32_t kPXfer = kPBytes + 128 * 4;          // ... followed by the 128 per-row integers
+constexpr uint32_t kPStride = 17 * 1024;                // distance between the two P buffers
+
+// ---- score CTA
+constexpr int kNumKSlots = 11;
+constexpr uint32_t kKSlotBytes = 2 * kBoxBytes;         // 128 keys x 64 columns
+constexpr uint32_t kOffQRope = 0;                       // 128 rows x 64 bf16, 128-byte swizzle
+constexpr uint32_t kOffStage = 128 * 64 * 2;            // 2 x kPStride
+constexpr uint32_t kOffK = kOffStage + 2 * kPStride;
+constexpr uint32_t kOffABars = kOffK + kNumKSlots * kKSlotBytes;
+// ---- value CTA
+constexpr int kNumVSlots = 5;
+constexpr uint32_t kVSlotBytes = 4 * kBoxBytes;         // 64 keys x 256 columns
+constexpr uint32_t kOffV = 0;
+constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;    // 2 x kPStride (P~ then N)
+constexpr uint32_t kOffFin = kOffP + 2 * kPStride;      // float2 [2][128] (1/(l*S16), lse)
+constexpr uint32_t kOffBBars = kOffFin + 2 * 128 * 8;
+constexpr uint32_t kBarBytes = 512;
+constexpr uint32_t kSmemA = kOffABars + kBarBytes;
+constexpr uint32_t kSmemB = kOffBBars + kBarBytes;
+constexpr uint32_t kSmemBytes = kSmemA > kSmemB ? kSmemA : kSmemB;
+static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
+static_assert(kOffK % 1024 == 0 && kOffStage % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 // tensor-memory columns
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kQCol = 0;            // score CTA: Q, 288 columns (two bf16 per column)
-constexpr uint32_t kSCol = 288;          // score CTA: S buffers, 2 x 64 columns
+constexpr uint32_t kQCol = 0;            // score CTA: latent part of Q, 256 columns (two bf16 per column)
+constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 columns
 // value CTA: O occupies columns 0..511
 
-// shared-memory layout (offsets from the 1024-aligned base); both CTAs allocate the larger of the two
-constexpr uint32_t kOffK = 0;                                          // score CTA
-constexpr uint32_t kOffABars = kNumKStages * kKStageBytes;             // 221184
-constexpr uint32_t kOffV = 0;                                          // value CTA
-constexpr uint32_t kOffP = kNumVStages * kVStageBytes;                 // 131072
-constexpr uint32_t kOffN = kOffP + 2 * kPBytes;                        // int32 [2][128]
-constexpr uint32_t kOffFin = kOffN + 2 * 128 * 4;                      // float2 [2][128] (1/(l*S16), lse)
-constexpr uint32_t kOffBBars = kOffFin + 2 * 128 * 8;
-constexpr uint32_t kBarBytes = 256;
-constexpr uint32_t kSmemA = kOffABars + kBarBytes;
-constexpr uint32_t kSmemB = kOffBBars + kBarBytes;
-constexpr uint32_t kSmemBytes = (kSmemA > kSmemB ? kSmemA : kSmemB) + 1024;
-
 // barrier indices, score CTA
-enum { A_KFULL = 0, A_KEMPTY = A_KFULL + kNumKStages, A_SFULL = A_KEMPTY + kNumKStages, A_SEMPTY = A_SFULL + 2,
-       A_PEMPTY = A_SEMPTY + 2, A_QREADY = A_PEMPTY + 2, A_QFREE, A_NUM };
+enum { A_KFULL = 0, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2,
+       A_PEMPTY = A_SEMPTY + 2, A_PSTAGED = A_PEMPTY + 2, A_QREADY = A_PSTAGED + 2, A_QFREE, A_NUM };
 // barrier indices, value CTA
-enum { B_VFULL = 0, B_VEMPTY = B_VFULL + kNumVStages, B_PFULL = B_VEMPTY + kNumVStages, B_OREADY = B_PFULL + 2,
+enum { B_VFULL = 0, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + 2,
        B_PVDONE = B_OREADY + 2, B_FINFULL = B_PVDONE + 2, B_NUM = B_FINFULL + 2 };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
 
@@ -97,17 +106,28 @@ struct UnitIter {
 
 __device__ __forceinline__ void report_timeout(int* status) { atomicExch(status, kStatusTimeout); }
 
+// Wait whose verdict is the same in every lane of the warp, so that the warp-collective tensor-memory
+// instructions that follow are never executed by a part of it.
+template <bool kClusterAcquire = false>
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, mbar_wait<kClusterAcquire>(bar, parity));
+}
+
 }  // namespace
 
 template <int kMode, bool kGuard>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams prm) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
   const bool is_score = rank == 0;
   const int part = blockIdx.x >> 1;
+  if (smem_base & 1023u) {   // the swizzled tiles assume a 1024-byte aligned window; identical in both CTAs
+    if (tid == 0) report_timeout(prm.status);
+    return;
+  }
 
   const uint32_t bars = smem_base + (is_score ? kOffABars : kOffBBars);
   auto bar = [&](int i) { return bars + 8u * i; };
@@ -119,14 +139,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
 
   if (tid == 0) {
     if (is_score) {
-      for (int i = 0; i < kNumKStages; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
-      for (int i = 0; i < 2; ++i) { mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 128); mbar_init(bar(A_PEMPTY + i), 1); }
+      for (int i = 0; i < kNumKSlots; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 128);
+        mbar_init(bar(A_PEMPTY + i), 1); mbar_init(bar(A_PSTAGED + i), 128);
+      }
       mbar_init(bar(A_QREADY), 128);
       mbar_init(bar(A_QFREE), 1);
     } else {
-      for (int i = 0; i < kNumVStages; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
+      for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
       for (int i = 0; i < 2; ++i) {
-        mbar_init(bar(B_PFULL + i), 128); mbar_init(bar(B_OREADY + i), 128);
+        mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 128);
         mbar_init(bar(B_PVDONE + i), 1); mbar_init(bar(B_FINFULL + i), 128);
       }
     }
@@ -139,25 +162,28 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
   cluster_arrive();
   cluster_wait();          // peer barriers are initialised before anyone signals them
   tc_fence_after_sync();
-  uint32_t tbase;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tbase) : "r"(tmem_slot));
+  const uint32_t tbase = ld_shared_b32(tmem_slot);
   if (tid == 0) AMLA_STAMP(prm, part, is_score ? 0 : 1, 0);
 
   bool ok = true;
   UnitIter iter(prm, part);
   Unit u;
-  uint32_t gt = 0;      // tiles processed by this cluster so far (all roles count identically)
+  uint32_t gt = 0;      // 64-key pages processed by this cluster so far (all roles count identically)
   uint32_t un = 0;      // units processed so far
 
   if (is_score) {
     // ======================================================================= score CTA
+    uint32_t gs = 0;    // score tiles (one or two pages) so far
+    uint32_t gc = 0;    // K ring slots so far
     if (wid < 4) {
       // ---- softmax warpgroup: thread = query row
       const int r = tid;
       const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+      const bool scale_nonneg = prm.scale_log2 >= 0.f;
+      const uint32_t mask_fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
       while (ok && iter.next(u)) {
-        // Q row -> tensor memory (previous unit's QK^T must be finished with it)
-        ok = mbar_wait(bar(A_QFREE), (un & 1) ^ 1);
+        // Q row -> tensor memory / shared memory (the previous unit's QK^T must be finished with it)
+        ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
         if (!ok) break;
         tc_fence_after_sync();
         if (tid == 0) AMLA_STAMP(prm, part, 10, un);
@@ -165,16 +191,25 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
           const bool valid = r < u.nrows;
           const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDqk);
 #pragma unroll 1
-          for (int blk = 0; blk < 9; ++blk) {
-            uint32_t regs[32];
+          for (int blk = 0; blk < 8; blk += 2) {
+            uint32_t r0[32], r1[32];
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-              uint4 v = valid ? __ldg(qrow + blk * 8 + c) : make_uint4(0, 0, 0, 0);
-              regs[4 * c] = v.x; regs[4 * c + 1] = v.y; regs[4 * c + 2] = v.z; regs[4 * c + 3] = v.w;
+              const uint4 v = valid ? __ldg(qrow + blk * 8 + c) : make_uint4(0, 0, 0, 0);
+              r0[4 * c] = v.x; r0[4 * c + 1] = v.y; r0[4 * c + 2] = v.z; r0[4 * c + 3] = v.w;
+              const uint4 w = valid ? __ldg(qrow + blk * 8 + 8 + c) : make_uint4(0, 0, 0, 0);
+              r1[4 * c] = w.x; r1[4 * c + 1] = w.y; r1[4 * c + 2] = w.z; r1[4 * c + 3] = w.w;
             }
-            tmem_st_32x32b_x32(tbase + lane_base + kQCol + blk * 32, regs);
+            tmem_st_32x32b_x32(tbase + lane_base + kQCol + blk * 32, r0);
+            tmem_st_32x32b_x32(tbase + lane_base + kQCol + blk * 32 + 32, r1);
+          }
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint4 v = valid ? __ldg(qrow + 64 + c) : make_uint4(0, 0, 0, 0);
+            st_shared_v4(smem_base + kOffQRope + sw128_offset(r, c), v.x, v.y, v.z, v.w);
           }
           tmem_wait_st();
+          fence_proxy_async_smem();
         }
         tc_fence_before_sync();
         mbar_arrive(bar(A_QREADY));
@@ -183,87 +218,110 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
         RowState st;
         row_state_init(st);
         const int tok = (u.r0 + r) / prm.H;
-        const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);   // keys 0..visible-1 are seen by this row
-        const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // tiles from here on may hold hidden keys
-        const bool scale_nonneg = prm.scale_log2 >= 0.f;
+        const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);          // keys 0..visible-1 are seen by this row
+        const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // pages from here on may hold hidden keys
 
-        for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
-          const uint32_t s = gt & 1, k = gt >> 1;
-          ok = mbar_wait(bar(A_SFULL + s), k & 1);
+        for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
+          const int npages = min(2, u.t1 - t);
+          const uint32_t sb = gs & 1;
+          ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
           if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
-          uint32_t a[64];
-          {
-            uint32_t lo[32], hi[32];
-            tmem_ld_32x32b_x32(tbase + lane_base + kSCol + 64 * s, lo);
-            tmem_ld_32x32b_x32(tbase + lane_base + kSCol + 64 * s + 32, hi);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) { a[i] = lo[i]; a[32 + i] = hi[i]; }
-          }
-          tc_fence_before_sync();
-          mbar_arrive(bar(A_SEMPTY + s));
-          if (tid == 0) AMLA_STAMP(prm, part, 6, gt);
+          const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
+          const bool masked = t + npages > first_masked_tile;
+          const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
 
-          // lines 5-6: mask, running max (taken on the raw scores; the scale is folded into the FMA below)
-          const int nvis = visible - t * kPage;            // keys of this tile the row sees (may be <= 0 or >= 64)
-          if (t >= first_masked_tile) {
-            const uint32_t fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
+          // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
+          float ext = scale_nonneg ? -INFINITY : INFINITY;
 #pragma unroll
-            for (int i = 0; i < 64; ++i) a[i] = (i < nvis) ? a[i] : fill;
-          }
-          float ext;
-          if (scale_nonneg) {
-            ext = -INFINITY;
+          for (int h = 0; h < 2; ++h) {
+            if (h < npages) {
+              uint32_t lo[32], hi[32];
+              tmem_ld_32x32b_x32(scol + 64 * h, lo);
+              tmem_ld_32x32b_x32(scol + 64 * h + 32, hi);
+              tmem_wait_ld();
+              if (masked) {
 #pragma unroll
-            for (int i = 0; i < 64; i += 2) ext = fmax3(ext, __uint_as_float(a[i]), __uint_as_float(a[i + 1]));
-          } else {
-            ext = INFINITY;
+                for (int i = 0; i < 32; ++i) {
+                  lo[i] = (64 * h + i < nvis) ? lo[i] : mask_fill;
+                  hi[i] = (64 * h + 32 + i < nvis) ? hi[i] : mask_fill;
+                }
+              }
+              if (scale_nonneg) {
 #pragma unroll
-            for (int i = 0; i < 64; i += 2) ext = fminf(ext, fminf(__uint_as_float(a[i]), __uint_as_float(a[i + 1])));
+                for (int i = 0; i < 32; ++i) ext = fmax3(ext, __uint_as_float(lo[i]), __uint_as_float(hi[i]));
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) ext = fminf(ext, fminf(__uint_as_float(lo[i]), __uint_as_float(hi[i])));
+              }
+            }
           }
           const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
           const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
-          // lines 6, 10: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
-          float rs0 = 0.f, rs1 = 0.f;
-          uint32_t pk[32];
           const float nsub = -sp.m2_sub;
-          if (t >= first_masked_tile) {
+          float rs0 = 0.f, rs1 = 0.f;
+
+          // lines 6, 10 per 64-key half: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
-              float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
-              p0 = (2 * i < nvis) ? p0 : 0.f;
-              p1 = (2 * i + 1 < nvis) ? p1 : 0.f;
-              rs0 += p0; rs1 += p1;
-              pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
-            }
-          } else {
+          for (int h = 0; h < 2; ++h) {
+            if (h < npages) {
+              uint32_t a[64];
+              {
+                uint32_t lo[32], hi[32];
+                tmem_ld_32x32b_x32(scol + 64 * h, lo);
+                tmem_ld_32x32b_x32(scol + 64 * h + 32, hi);
+                tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
-              const float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
-              rs0 += p0; rs1 += p1;
-              pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+                for (int i = 0; i < 32; ++i) { a[i] = lo[i]; a[32 + i] = hi[i]; }
+              }
+              if (h == npages - 1) {       // the score tile has been read for the last time
+                tc_fence_before_sync();
+                mbar_arrive(bar(A_SEMPTY + sb));
+                if (tid == 0) AMLA_STAMP(prm, part, 6, gt);
+              }
+              uint32_t pk[32];
+              if (masked) {
+                const int nv = nvis - 64 * h;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                  float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
+                  float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
+                  p0 = (2 * i < nv) ? p0 : 0.f;
+                  p1 = (2 * i + 1 < nv) ? p1 : 0.f;
+                  rs0 += p0; rs1 += p1;
+                  pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                  const float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
+                  const float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
+                  rs0 += p0; rs1 += p1;
+                  pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+                }
+              }
+              // stage P~ and N; the copy warp ships them to the value CTA
+              const uint32_t s = gt & 1, k = gt >> 1;
+              if (tid == 0) AMLA_STAMP(prm, part, 7, gt);
+              ok = warp_wait(bar(A_PEMPTY + s), (k & 1) ^ 1);
+              if (!ok) break;
+              if (tid == 0) AMLA_STAMP(prm, part, 8, gt);
+              const uint32_t stg = smem_base + kOffStage + s * kPStride;
+#pragma unroll
+              for (int c = 0; c < 8; ++c)
+                st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+              // the rescale (if any) belongs to the first half; the second half leaves O alone
+              const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
+                                                  : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
+              st_shared_b32(stg + kPBytes + r * 4, nword);
+              fence_proxy_async_smem();
+              mbar_arrive(bar(A_PSTAGED + s));
+              if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
+              ++gt;
             }
           }
           st.l = st.l * sp.l_up + (rs0 + rs1);
-
-          // hand P~ and N to the value CTA
-          if (tid == 0) AMLA_STAMP(prm, part, 7, gt);
-          ok = mbar_wait(bar(A_PEMPTY + s), (k & 1) ^ 1);
-          if (!ok) break;
-          if (tid == 0) AMLA_STAMP(prm, part, 8, gt);
-          const uint32_t pdst = peerB_base + kOffP + s * kPBytes;
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            st_cluster_v4(pdst + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-          const uint32_t nword = (kMode == 2) ? __float_as_uint(sp.l_up) : static_cast<uint32_t>(sp.n_bits);
-          st_cluster_b32(peerB_base + kOffN + (s * 128 + r) * 4, nword);
-          fence_proxy_async_all();
-          mbar_arrive_cluster(peerB_bars + 8u * (B_PFULL + s));
-          if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
         }
         if (!ok) break;
         // line 20 scalars: 1 / (l * S16) and lse = m + ln l
@@ -280,60 +338,81 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producer: K tiles (all 576 columns)
+      // ---- TMA producer: K, nine slots (64 columns each) per score tile
       if (lane == 0) {
         uint32_t issued = 0;
         while (ok && iter.next(u)) {
           const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
-          for (int t = u.t0; t < u.t1; ++t, ++gt) {
-            const uint32_t stg = gt % kNumKStages, rnd = gt / kNumKStages;
-            ok = mbar_wait(bar(A_KEMPTY + stg), (rnd & 1) ^ 1);
-            if (!ok) break;
-            AMLA_STAMP(prm, part, 2, gt);
-            const int page = __ldg(bt + t);
-            mbar_arrive_expect_tx(bar(A_KFULL + stg), kKStageBytes);
-            const uint32_t dst = smem_base + kOffK + stg * kKStageBytes;
-#pragma unroll
-            for (int c = 0; c < 9; ++c) tma_load_2d(dst + c * kBoxBytes, &kv_map, c * 64, page * kPage, bar(A_KFULL + stg));
-            ++issued;
+          for (int t = u.t0; t < u.t1 && ok; t += 2) {
+            const int npages = min(2, u.t1 - t);
+            const int page0 = __ldg(bt + t);
+            const int page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
+            for (int c = 0; c < 9; ++c, ++gc) {
+              const uint32_t slot = gc % kNumKSlots, rnd = gc / kNumKSlots;
+              ok = mbar_wait(bar(A_KEMPTY + slot), (rnd & 1) ^ 1);
+              if (!ok) break;
+              if (c == 0) AMLA_STAMP(prm, part, 2, gt);
+              AMLA_STAMP(prm, part, 20, gc);
+              mbar_arrive_expect_tx(bar(A_KFULL + slot), npages * kBoxBytes);
+              const uint32_t dst = smem_base + kOffK + slot * kKSlotBytes;
+              tma_load_2d(dst, &kv_map, c * 64, page0 * kPage, bar(A_KFULL + slot));
+              if (npages > 1) tma_load_2d(dst + kBoxBytes, &kv_map, c * 64, page1 * kPage, bar(A_KFULL + slot));
+              ++issued;
+            }
+            gt += npages;
           }
         }
         if (!ok) {
           report_timeout(prm.status);
           // let copies that are still in flight land before the CTA exits
-          for (uint32_t i = 0; i < kNumKStages && i < issued; ++i) {
+          for (uint32_t i = 0; i < kNumKSlots && i < issued; ++i) {
             const uint32_t n = issued - 1 - i;
-            mbar_wait(bar(A_KFULL + n % kNumKStages), (n / kNumKStages) & 1);
+            mbar_wait(bar(A_KFULL + n % kNumKSlots), (n / kNumKSlots) & 1);
           }
         }
       }
     } else if (wid == 5) {
-      // ---- MMA issuer: S[s] = Q K_t^T, 36 steps of K = 16
+      // ---- MMA issuer: S[sb] = Q K^T, 36 steps of K = 16 over nine slots
       if (lane == 0) {
-        constexpr uint32_t idesc = make_idesc_bf16(128, 64, false, false);
+        constexpr uint32_t idesc128 = make_idesc_bf16(128, 128, false, false);
+        constexpr uint32_t idesc64 = make_idesc_bf16(128, 64, false, false);
         while (ok && iter.next(u)) {
           ok = mbar_wait(bar(A_QREADY), un & 1);
           if (!ok) break;
           tc_fence_after_sync();
-          for (int t = u.t0; t < u.t1; ++t, ++gt) {
-            const uint32_t stg = gt % kNumKStages, rnd = gt / kNumKStages;
-            const uint32_t s = gt & 1, k = gt >> 1;
-            ok = mbar_wait(bar(A_KFULL + stg), rnd & 1);
-            if (!ok) break;
-            ok = mbar_wait(bar(A_SEMPTY + s), (k & 1) ^ 1);
+          for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
+            const int npages = min(2, u.t1 - t);
+            const uint32_t idesc = npages > 1 ? idesc128 : idesc64;
+            const uint32_t sb = gs & 1;
+            ok = mbar_wait(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
             AMLA_STAMP(prm, part, 3, gt);
-            const uint32_t kbase = smem_base + kOffK + stg * kKStageBytes;
-            const uint32_t d = tbase + kSCol + 64 * s;
+            const uint32_t d = tbase + kSCol + 128 * sb;
+            for (int c = 0; c < 9; ++c, ++gc) {
+              const uint32_t slot = gc % kNumKSlots, rnd = gc / kNumKSlots;
+              ok = mbar_wait(bar(A_KFULL + slot), rnd & 1);
+              if (!ok) break;
+              tc_fence_after_sync();
+              AMLA_STAMP(prm, part, 21, gc);
+              const uint32_t kbase = smem_base + kOffK + slot * kKSlotBytes;
 #pragma unroll
-            for (int ks = 0; ks < 36; ++ks) {
-              const uint64_t bd = make_smem_desc_sw128(kbase + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024);
-              mma_ts(d, tbase + kQCol + 8 * ks, bd, idesc, ks > 0);
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t bd = make_smem_desc_sw128(kbase + kk * 32, 16, 1024);
+                if (c < 8) {
+                  mma_ts(d, tbase + kQCol + 32 * c + 8 * kk, bd, idesc, (c | kk) != 0);
+                } else {
+                  const uint64_t ad = make_smem_desc_sw128(smem_base + kOffQRope + kk * 32, 16, 1024);
+                  mma_ss(d, ad, bd, idesc, 1u);
+                }
+              }
+              mma_commit(bar(A_KEMPTY + slot));
+              AMLA_STAMP(prm, part, 22, gc);
             }
-            mma_commit(bar(A_KEMPTY + stg));
-            mma_commit(bar(A_SFULL + s));
+            if (!ok) break;
+            mma_commit(bar(A_SFULL + sb));
             AMLA_STAMP(prm, part, 4, gt);
+            gt += npages;
           }
           if (!ok) break;
           mma_commit(bar(A_QFREE));
@@ -341,9 +420,26 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
         }
         if (!ok) report_timeout(prm.status);
       }
+    } else if (wid == 6) {
+      // ---- copy issuer: staged P~ / N of one half -> value CTA, counted on its PFULL barrier
+      if (lane == 0) {
+        while (ok && iter.next(u)) {
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            const uint32_t s = gt & 1, k = gt >> 1;
+            ok = mbar_wait(bar(A_PSTAGED + s), k & 1);
+            if (!ok) break;
+            const uint32_t pfull = peerB_bars + 8u * (B_PFULL + s);
+            AMLA_STAMP(prm, part, 23, gt);
+            mbar_arrive_expect_tx_cluster(pfull, kPXfer);
+            bulk_copy_to_cluster(peerB_base + kOffP + s * kPStride, smem_base + kOffStage + s * kPStride, kPXfer, pfull);
+          }
+        }
+        if (!ok) report_timeout(prm.status);
+      }
     }
   } else {
     // ======================================================================= value CTA
+    uint32_t gv = 0;    // V ring slots so far (two per page)
     if (wid < 4) {
       // ---- correction + epilogue warpgroup: thread = query row
       const int r = tid;
@@ -351,16 +447,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
       while (ok && iter.next(u)) {
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
           const uint32_t s = gt & 1, k = gt >> 1;
-          ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
+          ok = warp_wait(bar(B_PFULL + s), k & 1);
           if (!ok) break;
           if (tid == 0) AMLA_STAMP(prm, part, 13, gt);
-          uint32_t nword;
-          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(nword) : "r"(smem_base + kOffN + (s * 128 + r) * 4));
+          const uint32_t nword = ld_shared_b32(smem_base + kOffP + s * kPStride + kPBytes + r * 4);
           const bool mine = (kMode == 2) ? (__uint_as_float(nword) != 1.f) : (nword != 0u);
           if (__any_sync(0xffffffffu, mine) && t > u.t0) {
-            // lines 13-16: O <- AS_FP32(AS_INT32(O) + N), after P V of the previous tile has landed
+            // lines 13-16: O <- AS_FP32(AS_INT32(O) + N), after P V of the previous page has landed
             const uint32_t gp = gt - 1;
-            ok = mbar_wait(bar(B_PVDONE + (gp & 1)), (gp >> 1) & 1);
+            ok = warp_wait(bar(B_PVDONE + (gp & 1)), (gp >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
             // two 32-column chunks in flight: the load of one overlaps the arithmetic of the other
@@ -397,9 +492,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
         // ---- epilogue (line 20): out = O / (l * S16)
         {
           const uint32_t gl = gt - 1;
-          ok = mbar_wait(bar(B_PVDONE + (gl & 1)), (gl >> 1) & 1);
+          ok = warp_wait(bar(B_PVDONE + (gl & 1)), (gl >> 1) & 1);
           if (!ok) break;
-          ok = mbar_wait<true>(bar(B_FINFULL + (un & 1)), (un >> 1) & 1);
+          ok = warp_wait<true>(bar(B_FINFULL + (un & 1)), (un >> 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
           if (tid == 0) AMLA_STAMP(prm, part, 18, un);
@@ -449,29 +544,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producer: V tiles (first 512 columns of the same cache rows)
+      // ---- TMA producer: V, two slots (256 columns each) per page
       if (lane == 0) {
         uint32_t issued = 0;
         while (ok && iter.next(u)) {
           const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
-          for (int t = u.t0; t < u.t1; ++t, ++gt) {
-            const uint32_t stg = gt % kNumVStages, rnd = gt / kNumVStages;
-            ok = mbar_wait(bar(B_VEMPTY + stg), (rnd & 1) ^ 1);
-            if (!ok) break;
-            AMLA_STAMP(prm, part, 12, gt);
+          for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
             const int page = __ldg(bt + t);
-            mbar_arrive_expect_tx(bar(B_VFULL + stg), kVStageBytes);
-            const uint32_t dst = smem_base + kOffV + stg * kVStageBytes;
+            for (int nh = 0; nh < 2; ++nh, ++gv) {
+              const uint32_t slot = gv % kNumVSlots, rnd = gv / kNumVSlots;
+              ok = mbar_wait(bar(B_VEMPTY + slot), (rnd & 1) ^ 1);
+              if (!ok) break;
+              if (nh == 0) AMLA_STAMP(prm, part, 12, gt);
+              mbar_arrive_expect_tx(bar(B_VFULL + slot), kVSlotBytes);
+              const uint32_t dst = smem_base + kOffV + slot * kVSlotBytes;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) tma_load_2d(dst + c * kBoxBytes, &kv_map, c * 64, page * kPage, bar(B_VFULL + stg));
-            ++issued;
+              for (int c = 0; c < 4; ++c) tma_load_2d(dst + c * kBoxBytes, &kv_map, (nh * 4 + c) * 64, page * kPage, bar(B_VFULL + slot));
+              ++issued;
+            }
           }
         }
         if (!ok) {
           report_timeout(prm.status);
-          for (uint32_t i = 0; i < kNumVStages && i < issued; ++i) {
+          for (uint32_t i = 0; i < kNumVSlots && i < issued; ++i) {
             const uint32_t n = issued - 1 - i;
-            mbar_wait(bar(B_VFULL + n % kNumVStages), (n / kNumVStages) & 1);
+            mbar_wait(bar(B_VFULL + n % kNumVSlots), (n / kNumVSlots) & 1);
           }
         }
       }
@@ -480,30 +577,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
       if (lane == 0) {
         constexpr uint32_t idesc = make_idesc_bf16(128, 256, false, true);
         while (ok && iter.next(u)) {
-          for (int t = u.t0; t < u.t1; ++t, ++gt) {
-            const uint32_t stg = gt % kNumVStages, rnd = gt / kNumVStages;
+          for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
             const uint32_t s = gt & 1, k = gt >> 1;
-            ok = mbar_wait(bar(B_VFULL + stg), rnd & 1);
-            if (!ok) break;
-            ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
+            ok = mbar_wait(bar(B_PFULL + s), k & 1);
             if (!ok) break;
             ok = mbar_wait(bar(B_OREADY + s), k & 1);
             if (!ok) break;
-            fence_proxy_async_all();
-            tc_fence_after_sync();
-            AMLA_STAMP(prm, part, 15, gt);
-            const uint32_t vbase = smem_base + kOffV + stg * kVStageBytes;
-            const uint32_t pbase = smem_base + kOffP + s * kPBytes;
+            const uint32_t pbase = smem_base + kOffP + s * kPStride;
 #pragma unroll
-            for (int nh = 0; nh < 2; ++nh) {
+            for (int nh = 0; nh < 2; ++nh, ++gv) {
+              const uint32_t slot = gv % kNumVSlots, rnd = gv / kNumVSlots;
+              ok = ok && mbar_wait(bar(B_VFULL + slot), rnd & 1);
+              if (ok) {
+                tc_fence_after_sync();
+                if (nh == 0) AMLA_STAMP(prm, part, 15, gt);
+                const uint32_t vbase = smem_base + kOffV + slot * kVSlotBytes;
 #pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                const uint64_t ad = make_smem_desc_sw128(pbase + kk * 32, 16, 1024);
-                const uint64_t bd = make_smem_desc_sw128(vbase + nh * 4 * kBoxBytes + kk * 2048, kBoxBytes, 1024);
-                mma_ss(tbase + nh * 256, ad, bd, idesc, (t > u.t0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < 4; ++kk) {
+                  const uint64_t ad = make_smem_desc_sw128(pbase + kk * 32, 16, 1024);
+                  const uint64_t bd = make_smem_desc_sw128(vbase + kk * 2048, kBoxBytes, 1024);
+                  mma_ss(tbase + nh * 256, ad, bd, idesc, (t > u.t0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(bar(B_VEMPTY + slot));
               }
             }
-            mma_commit(bar(B_VEMPTY + stg));
+            if (!ok) break;
             mma_commit(bar(B_PVDONE + s));
             AMLA_STAMP(prm, part, 16, gt);
           }
