@@ -104,6 +104,24 @@ struct UnitIter {
   }
 };
 
+// Finds the unit that holds the k-th page (kTiles = false) or the k-th score tile (kTiles = true) of this
+// cluster's part; k never decreases between calls.  Used by producer lanes that advance independently.
+template <bool kTiles>
+struct Cursor {
+  UnitIter it;
+  Unit u;
+  int base;      // index of the current unit's first page / score tile
+  bool valid;
+  __device__ Cursor(const DecodeParams& prm, int part) : it(prm, part), base(0) { valid = it.next(u); }
+  __device__ int count() const { return kTiles ? (u.t1 - u.t0 + 1) / 2 : (u.t1 - u.t0); }
+  // false when k lies beyond the part's work; otherwise `local` is the index within the unit
+  __device__ bool locate(int k, int& local) {
+    while (valid && k >= base + count()) { base += count(); valid = it.next(u); }
+    local = k - base;
+    return valid;
+  }
+};
+
 __device__ __forceinline__ void report_timeout(int* status) { atomicExch(status, kStatusTimeout); }
 
 // Wait whose verdict is the same in every lane of the warp, so that the warp-collective tensor-memory
@@ -117,7 +135,7 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
 
 template <int kMode, bool kGuard>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams prm) {
+decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap v_map, const DecodeParams prm) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t smem_base = smem_u32(smem_raw);
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
@@ -155,6 +173,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
     }
     fence_mbar_init();
     prefetch_tensormap(&kv_map);
+    prefetch_tensormap(&v_map);
   }
   if (wid == 5) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
   tc_fence_before_sync();
@@ -338,37 +357,49 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producer: K, nine slots (64 columns each) per score tile
-      if (lane == 0) {
-        uint32_t issued = 0;
-        while (ok && iter.next(u)) {
-          const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
-          for (int t = u.t0; t < u.t1 && ok; t += 2) {
-            const int npages = min(2, u.t1 - t);
-            const int page0 = __ldg(bt + t);
-            const int page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
-            for (int c = 0; c < 9; ++c, ++gc) {
-              const uint32_t slot = gc % kNumKSlots, rnd = gc / kNumKSlots;
-              ok = mbar_wait(bar(A_KEMPTY + slot), (rnd & 1) ^ 1);
-              if (!ok) break;
-              if (c == 0) AMLA_STAMP(prm, part, 2, gt);
-              AMLA_STAMP(prm, part, 20, gc);
-              mbar_arrive_expect_tx(bar(A_KFULL + slot), npages * kBoxBytes);
-              const uint32_t dst = smem_base + kOffK + slot * kKSlotBytes;
-              tma_load_2d(dst, &kv_map, c * 64, page0 * kPage, bar(A_KFULL + slot));
-              if (npages > 1) tma_load_2d(dst + kBoxBytes, &kv_map, c * 64, page1 * kPage, bar(A_KFULL + slot));
-              ++issued;
+      // ---- TMA producers: K, nine slots (64 columns each) per score tile.  Lane l owns ring slot l and loads
+      // every kNumKSlots-th slot of the sequence; the lanes poll without blocking, so that a slot that is
+      // still in use never holds up the loads of the others (one thread issuing the ring in order reaches
+      // a quarter of the rate).
+      {
+        Cursor<true> cur(prm, part);
+        int my_gc = lane;                       // next slot of the sequence this lane loads
+        bool fin = lane >= kNumKSlots, have = false;
+        int page0 = 0, page1 = 0, npages = 0, c = 0;
+        int issued = 0;
+        const uint64_t t_start = global_timer_ns();
+        for (uint32_t spin = 0;; ++spin) {
+          if (!fin && !have) {
+            int lt;
+            if (cur.locate(my_gc / 9, lt)) {
+              const int t = cur.u.t0 + 2 * lt;
+              const int32_t* bt = prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq;
+              npages = min(2, cur.u.t1 - t);
+              page0 = __ldg(bt + t);
+              page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
+              c = my_gc % 9;
+              have = true;
+            } else {
+              fin = true;
             }
-            gt += npages;
           }
+          if (have && mbar_probe(bar(A_KEMPTY + lane), (((my_gc / kNumKSlots) & 1) ^ 1))) {
+            AMLA_STAMP(prm, part, 20, my_gc);
+            mbar_arrive_expect_tx(bar(A_KFULL + lane), npages * kBoxBytes);
+            const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
+            tma_load_2d(dst, &kv_map, c * 64, page0 * kPage, bar(A_KFULL + lane));
+            if (npages > 1) tma_load_2d(dst + kBoxBytes, &kv_map, c * 64, page1 * kPage, bar(A_KFULL + lane));
+            my_gc += kNumKSlots;
+            ++issued;
+            have = false;
+          }
+          if (__all_sync(0xffffffffu, fin)) break;
+          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > 4 * kWaitLimitNs)) { ok = false; break; }
         }
         if (!ok) {
-          report_timeout(prm.status);
-          // let copies that are still in flight land before the CTA exits
-          for (uint32_t i = 0; i < kNumKSlots && i < issued; ++i) {
-            const uint32_t n = issued - 1 - i;
-            mbar_wait(bar(A_KFULL + n % kNumKSlots), (n / kNumKSlots) & 1);
-          }
+          if (lane == 0) report_timeout(prm.status);
+          // let the copy that may still be in flight land before the CTA exits
+          if (issued > 0 && lane < kNumKSlots) mbar_wait(bar(A_KFULL + lane), (issued - 1) & 1);
         }
       }
     } else if (wid == 5) {
@@ -544,32 +575,38 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const DecodeParams 
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producer: V, two slots (256 columns each) per page
-      if (lane == 0) {
-        uint32_t issued = 0;
-        while (ok && iter.next(u)) {
-          const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
-          for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
-            const int page = __ldg(bt + t);
-            for (int nh = 0; nh < 2; ++nh, ++gv) {
-              const uint32_t slot = gv % kNumVSlots, rnd = gv / kNumVSlots;
-              ok = mbar_wait(bar(B_VEMPTY + slot), (rnd & 1) ^ 1);
-              if (!ok) break;
-              if (nh == 0) AMLA_STAMP(prm, part, 12, gt);
-              mbar_arrive_expect_tx(bar(B_VFULL + slot), kVSlotBytes);
-              const uint32_t dst = smem_base + kOffV + slot * kVSlotBytes;
-#pragma unroll
-              for (int c = 0; c < 4; ++c) tma_load_2d(dst + c * kBoxBytes, &kv_map, (nh * 4 + c) * 64, page * kPage, bar(B_VFULL + slot));
-              ++issued;
+      // ---- TMA producers: V, two slots (256 columns each, one 3-D box) per page; lane l owns ring slot l
+      {
+        Cursor<false> cur(prm, part);
+        int my_gv = lane;
+        bool fin = lane >= kNumVSlots, have = false;
+        int page = 0;
+        int issued = 0;
+        const uint64_t t_start = global_timer_ns();
+        for (uint32_t spin = 0;; ++spin) {
+          if (!fin && !have) {
+            int lt;
+            if (cur.locate(my_gv / 2, lt)) {
+              page = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + cur.u.t0 + lt);
+              have = true;
+            } else {
+              fin = true;
             }
           }
+          if (have && mbar_probe(bar(B_VEMPTY + lane), (((my_gv / kNumVSlots) & 1) ^ 1))) {
+            if ((my_gv & 1) == 0) AMLA_STAMP(prm, part, 12, my_gv / 2);
+            mbar_arrive_expect_tx(bar(B_VFULL + lane), kVSlotBytes);
+            tma_load_3d(smem_base + kOffV + lane * kVSlotBytes, &v_map, 0, page * kPage, (my_gv & 1) * 4, bar(B_VFULL + lane));
+            my_gv += kNumVSlots;
+            ++issued;
+            have = false;
+          }
+          if (__all_sync(0xffffffffu, fin)) break;
+          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > 4 * kWaitLimitNs)) { ok = false; break; }
         }
         if (!ok) {
-          report_timeout(prm.status);
-          for (uint32_t i = 0; i < kNumVSlots && i < issued; ++i) {
-            const uint32_t n = issued - 1 - i;
-            mbar_wait(bar(B_VFULL + n % kNumVSlots), (n / kNumVSlots) & 1);
-          }
+          if (lane == 0) report_timeout(prm.status);
+          if (issued > 0 && lane < kNumVSlots) mbar_wait(bar(B_VFULL + lane), (issued - 1) & 1);
         }
       }
     } else if (wid == 5) {
@@ -656,7 +693,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 template <int kMode, bool kGuard>
-cudaError_t launch_variant(const CUtensorMap& map, const DecodeParams& prm, cudaStream_t stream) {
+cudaError_t launch_variant(const CUtensorMap& map, const CUtensorMap& vmap, const DecodeParams& prm, cudaStream_t stream) {
   auto kern = decode_tc_kernel<kMode, kGuard>;
   // the opt-in to large dynamic shared memory is per device and per kernel; do it once each
   static std::atomic<uint64_t> done{0};
@@ -669,7 +706,7 @@ cudaError_t launch_variant(const CUtensorMap& map, const DecodeParams& prm, cuda
     if (err != cudaSuccess) return err;
     done.fetch_or(bit, std::memory_order_release);
   }
-  kern<<<2 * prm.P, kThreads, kSmemBytes, stream>>>(map, prm);
+  kern<<<2 * prm.P, kThreads, kSmemBytes, stream>>>(map, vmap, prm);
   return cudaGetLastError();
 }
 
@@ -691,11 +728,24 @@ cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* 
                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  // V: the same rows seen as (64 columns, rows, column block); one box = 64 keys x 4 column blocks, laid out in
+  // shared memory as [column block][key][64 columns] -- four of the 2-D boxes above in one instruction.
+  CUtensorMap vmap;
+  {
+    const cuuint64_t vdims[3] = {64, static_cast<cuuint64_t>(prm.num_blocks) * kPage, static_cast<cuuint64_t>(kDqk / 64)};
+    const cuuint64_t vstrides[2] = {static_cast<cuuint64_t>(kDqk) * 2, 128};
+    const cuuint32_t vbox[3] = {64, 64, 4};
+    const cuuint32_t vestr[3] = {1, 1, 1};
+    const CUresult vr = encode(&vmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(prm.kv), vdims, vstrides,
+                               vbox, vestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (vr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
   const int mode = prm.flags & 3;
   const bool guard = !(prm.flags & 4);
-  if (mode == 0) return guard ? launch_variant<0, true>(map, prm, stream) : launch_variant<0, false>(map, prm, stream);
-  if (mode == 1) return guard ? launch_variant<1, true>(map, prm, stream) : launch_variant<1, false>(map, prm, stream);
-  return launch_variant<2, true>(map, prm, stream);
+  if (mode == 0) return guard ? launch_variant<0, true>(map, vmap, prm, stream) : launch_variant<0, false>(map, vmap, prm, stream);
+  if (mode == 1) return guard ? launch_variant<1, true>(map, vmap, prm, stream) : launch_variant<1, false>(map, vmap, prm, stream);
+  return launch_variant<2, true>(map, vmap, prm, stream);
 }
 
 }  // namespace amla
