@@ -44,7 +44,7 @@ struct DecodeParams {
 
 // Optional per-role timeline (compiled in with -DAMLA_TRACE only): every stamp is the SM's cycle
 // counter, stored at trace[(part * kTraceEvents + event) * kTraceTiles + index].
-constexpr int kTraceEvents = 24;
+constexpr int kTraceEvents = 32;
 constexpr int kTraceTiles = 96;
 #ifdef AMLA_TRACE
 #define AMLA_STAMP(prm, part, ev, idx)                                                                      \

@@ -4,8 +4,8 @@
 //
 //   score CTA (cluster rank 0)   the 512 latent columns of Q (128 x 512 bf16) are resident in tensor
 //       memory as the A operand, the 64 RoPE columns in shared memory.  K arrives by TMA in slots of
-//       128 keys x 64 columns (two pages stacked), nine slots per score tile, through an 11-slot
-//       ring; S = Q K^T (128 x 128, FP32) by tcgen05.mma into a double-buffered TMEM tile.  The
+//       128 keys x 192 columns (two pages stacked, one 4-D box each), three slots per score tile,
+//       through a ring; S = Q K^T (128 x 128, FP32) by tcgen05.mma into a double-buffered TMEM tile.  The
 //       softmax warpgroup runs Algorithm 2's per-row recurrence (lines 5-12) once per score tile,
 //       writes the bf16 probabilities P~ = bf16(P * S16) of each 64-key half plus the per-row integer
 //       N into a local staging buffer, and a bulk shared-to-shared copy moves it into the value CTA.
@@ -32,15 +32,21 @@ using namespace sm100;
 
 namespace {
 
+#ifdef AMLA_TRACE
+constexpr int kThreads = 256;            // trace builds add warp 7, which watches the K slots fill
+#else
 constexpr int kThreads = 224;            // warps 0-3: softmax / correction, 4: TMA, 5: MMA + TMEM alloc, 6: copy / relay
+#endif
 constexpr uint32_t kBoxBytes = 64 * 64 * 2;             // one 64-key x 64-column TMA box
 constexpr uint32_t kPBytes = 128 * 64 * 2;              // P~ of one 64-key half: 128 rows x 128 B
 constexpr uint32_t kPXfer = kPBytes + 128 * 4;          // ... followed by the 128 per-row integers
 constexpr uint32_t kPStride = 17 * 1024;                // distance between the two P buffers
 
 // ---- score CTA
-constexpr int kNumKSlots = 11;
-constexpr uint32_t kKSlotBytes = 2 * kBoxBytes;         // 128 keys x 64 columns
+constexpr int kNumKSlots = 3;
+constexpr uint32_t kKPageBytes = 3 * kBoxBytes;         // 64 keys x 3 column blocks: [8 row groups][3 blocks][8 rows][128 B]
+constexpr uint32_t kKSlotBytes = 2 * kKPageBytes;       // 128 keys x 192 columns (two pages stacked)
+constexpr uint32_t kKGroupStride = 3 * 1024;            // distance between 8-row groups inside a slot
 constexpr uint32_t kOffQRope = 0;                       // 128 rows x 64 bf16, 128-byte swizzle
 constexpr uint32_t kOffStage = 128 * 64 * 2;            // 2 x kPStride
 constexpr uint32_t kOffK = kOffStage + 2 * kPStride;
@@ -253,7 +259,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
 
           // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
           float ext = scale_nonneg ? -INFINITY : INFINITY;
-#pragma unroll
+#pragma unroll 1
           for (int h = 0; h < 2; ++h) {
             if (h < npages) {
               uint32_t lo[32], hi[32];
@@ -282,7 +288,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           float rs0 = 0.f, rs1 = 0.f;
 
           // lines 6, 10 per 64-key half: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
-#pragma unroll
+#pragma unroll 1
           for (int h = 0; h < 2; ++h) {
             if (h < npages) {
               uint32_t a[64];
@@ -357,39 +363,43 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producers: K, nine slots (64 columns each) per score tile.  Lane l owns ring slot l and loads
-      // every kNumKSlots-th slot of the sequence; the lanes poll without blocking, so that a slot that is
-      // still in use never holds up the loads of the others (one thread issuing the ring in order reaches
-      // a quarter of the rate).
+      // ---- TMA producers: K, three slots (192 columns each) per score tile.  Lane l owns ring slot l and
+      // loads every kNumKSlots-th slot of the sequence; the lanes poll without blocking, so that a slot that
+      // is still in use never holds up the loads of the others (one thread issuing a ring in order reaches a
+      // fraction of the rate).
       {
         Cursor<true> cur(prm, part);
-        int my_gc = lane;                       // next slot of the sequence this lane loads
+        int my_tile = lane / 3, g = lane % 3;   // score tile and column-block group of the next slot this lane loads
+        uint32_t par = 1;                       // parity of the "empty" phase it has to see first
         bool fin = lane >= kNumKSlots, have = false;
-        int page0 = 0, page1 = 0, npages = 0, c = 0;
+        int page0 = 0, page1 = 0, npages = 0;
         int issued = 0;
+        const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane);
+        const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
         const uint64_t t_start = global_timer_ns();
         for (uint32_t spin = 0;; ++spin) {
           if (!fin && !have) {
             int lt;
-            if (cur.locate(my_gc / 9, lt)) {
+            if (cur.locate(my_tile, lt)) {
               const int t = cur.u.t0 + 2 * lt;
               const int32_t* bt = prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq;
               npages = min(2, cur.u.t1 - t);
               page0 = __ldg(bt + t);
               page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
-              c = my_gc % 9;
               have = true;
             } else {
               fin = true;
             }
           }
-          if (have && mbar_probe(bar(A_KEMPTY + lane), (((my_gc / kNumKSlots) & 1) ^ 1))) {
-            AMLA_STAMP(prm, part, 20, my_gc);
-            mbar_arrive_expect_tx(bar(A_KFULL + lane), npages * kBoxBytes);
-            const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
-            tma_load_2d(dst, &kv_map, c * 64, page0 * kPage, bar(A_KFULL + lane));
-            if (npages > 1) tma_load_2d(dst + kBoxBytes, &kv_map, c * 64, page1 * kPage, bar(A_KFULL + lane));
-            my_gc += kNumKSlots;
+          if (have && mbar_probe(my_empty, par)) {
+            AMLA_STAMP(prm, part, 20, issued * kNumKSlots + lane);
+            mbar_arrive_expect_tx(my_full, npages * kKPageBytes);
+            tma_load_4d(dst, &kv_map, 0, 0, 3 * g, page0 * 8, my_full);
+            if (npages > 1) tma_load_4d(dst + kKPageBytes, &kv_map, 0, 0, 3 * g, page1 * 8, my_full);
+            // kNumKSlots slots further on
+            g += kNumKSlots % 3; my_tile += kNumKSlots / 3;
+            if (g >= 3) { g -= 3; my_tile += 1; }
+            par ^= 1;
             ++issued;
             have = false;
           }
@@ -399,14 +409,21 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         if (!ok) {
           if (lane == 0) report_timeout(prm.status);
           // let the copy that may still be in flight land before the CTA exits
-          if (issued > 0 && lane < kNumKSlots) mbar_wait(bar(A_KFULL + lane), (issued - 1) & 1);
+          if (issued > 0 && lane < kNumKSlots) mbar_wait(my_full, (issued - 1) & 1);
         }
       }
     } else if (wid == 5) {
-      // ---- MMA issuer: S[sb] = Q K^T, 36 steps of K = 16 over nine slots
+      // ---- MMA issuer: S[sb] = Q K^T, 36 steps of K = 16 over three slots.  One thread runs this loop, so
+      // it is kept free of divisions and descriptor arithmetic: ring position, barrier addresses and the
+      // low descriptor word are stepped incrementally.
       if (lane == 0) {
         constexpr uint32_t idesc128 = make_idesc_bf16(128, 128, false, false);
         constexpr uint32_t idesc64 = make_idesc_bf16(128, 64, false, false);
+        constexpr uint32_t dhi = smem_desc_hi_sw128(kKGroupStride);
+        constexpr uint32_t qhi = smem_desc_hi_sw128(1024);
+        const uint32_t klo0 = smem_desc_lo(smem_base + kOffK, 16);
+        const uint32_t qlo0 = smem_desc_lo(smem_base + kOffQRope, 16);
+        uint32_t slot = 0, kpar = 0;          // ring position and the parity its "full" barrier completes next
         while (ok && iter.next(u)) {
           ok = mbar_wait(bar(A_QREADY), un & 1);
           if (!ok) break;
@@ -420,25 +437,33 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             tc_fence_after_sync();
             AMLA_STAMP(prm, part, 3, gt);
             const uint32_t d = tbase + kSCol + 128 * sb;
-            for (int c = 0; c < 9; ++c, ++gc) {
-              const uint32_t slot = gc % kNumKSlots, rnd = gc / kNumKSlots;
-              ok = mbar_wait(bar(A_KFULL + slot), rnd & 1);
+            uint32_t qa = tbase + kQCol;          // A operand: eight tensor-memory columns per K = 16 step
+            uint32_t acc = 0;
+#pragma unroll 1
+            for (int g = 0; g < 3; ++g) {
+              AMLA_STAMP(prm, part, 25, gc);
+              ok = mbar_wait(bar(A_KFULL) + 8 * slot, kpar);
               if (!ok) break;
               tc_fence_after_sync();
               AMLA_STAMP(prm, part, 21, gc);
-              const uint32_t kbase = smem_base + kOffK + slot * kKSlotBytes;
-#pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                const uint64_t bd = make_smem_desc_sw128(kbase + kk * 32, 16, 1024);
-                if (c < 8) {
-                  mma_ts(d, tbase + kQCol + 32 * c + 8 * kk, bd, idesc, (c | kk) != 0);
-                } else {
-                  const uint64_t ad = make_smem_desc_sw128(smem_base + kOffQRope + kk * 32, 16, 1024);
-                  mma_ss(d, ad, bd, idesc, 1u);
-                }
+              uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
+              const int n_ts = g < 2 ? 12 : 8;     // the last four steps take the RoPE columns of Q from shared memory
+#pragma unroll 1
+              for (int i = 0; i < n_ts; ++i) {
+                mma_ts(d, qa, smem_desc_join(klo, dhi), idesc, acc);
+                acc = 1;
+                qa += 8;
+                klo += ((i & 3) == 3) ? 64 - 6 : 2;   // next K step inside the block, or on to the next column block
               }
-              mma_commit(bar(A_KEMPTY + slot));
+              if (g == 2) {
+#pragma unroll 1
+                for (int kk = 0; kk < 4; ++kk) mma_ss(d, smem_desc_join(qlo0 + 2 * kk, qhi), smem_desc_join(klo + 2 * kk, dhi), idesc, 1u);
+              }
+              AMLA_STAMP(prm, part, 26, gc);
+              mma_commit(bar(A_KEMPTY) + 8 * slot);
               AMLA_STAMP(prm, part, 22, gc);
+              ++gc;
+              if (++slot == kNumKSlots) { slot = 0; kpar ^= 1; }
             }
             if (!ok) break;
             mma_commit(bar(A_SFULL + sb));
@@ -451,6 +476,25 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         }
         if (!ok) report_timeout(prm.status);
       }
+#ifdef AMLA_TRACE
+    } else if (wid == 7) {
+      // trace builds: lane l watches K slot l and stamps the arrival of its data (non-blocking polls)
+      if (prm.trace) {
+        Cursor<true> cur(prm, part);
+        int total = 0, lt;
+        while (cur.valid) { total += cur.count(); cur.locate(total, lt); }
+        total *= 3;
+        uint32_t par = 0;
+        int g = lane;
+        const uint64_t t_start = global_timer_ns();
+        for (uint32_t spin = 0;; ++spin) {
+          const bool act = lane < kNumKSlots && g < total;
+          if (act && mbar_probe(bar(A_KFULL + lane), par)) { AMLA_STAMP(prm, part, 24, g); g += kNumKSlots; par ^= 1; }
+          if (!__any_sync(0xffffffffu, act)) break;
+          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) break;
+        }
+      }
+#endif
     } else if (wid == 6) {
       // ---- copy issuer: staged P~ / N of one half -> value CTA, counted on its PFULL barrier
       if (lane == 0) {
@@ -578,26 +622,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       // ---- TMA producers: V, two slots (256 columns each, one 3-D box) per page; lane l owns ring slot l
       {
         Cursor<false> cur(prm, part);
-        int my_gv = lane;
+        int my_gv = lane;                       // next slot of the sequence this lane loads (page = gv / 2)
+        uint32_t par = 1;
         bool fin = lane >= kNumVSlots, have = false;
         int page = 0;
         int issued = 0;
+        const uint32_t my_full = bar(B_VFULL + lane), my_empty = bar(B_VEMPTY + lane);
+        const uint32_t dst = smem_base + kOffV + lane * kVSlotBytes;
         const uint64_t t_start = global_timer_ns();
         for (uint32_t spin = 0;; ++spin) {
           if (!fin && !have) {
             int lt;
-            if (cur.locate(my_gv / 2, lt)) {
+            if (cur.locate(my_gv >> 1, lt)) {
               page = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + cur.u.t0 + lt);
               have = true;
             } else {
               fin = true;
             }
           }
-          if (have && mbar_probe(bar(B_VEMPTY + lane), (((my_gv / kNumVSlots) & 1) ^ 1))) {
-            if ((my_gv & 1) == 0) AMLA_STAMP(prm, part, 12, my_gv / 2);
-            mbar_arrive_expect_tx(bar(B_VFULL + lane), kVSlotBytes);
-            tma_load_3d(smem_base + kOffV + lane * kVSlotBytes, &v_map, 0, page * kPage, (my_gv & 1) * 4, bar(B_VFULL + lane));
+          if (have && mbar_probe(my_empty, par)) {
+            if ((my_gv & 1) == 0) AMLA_STAMP(prm, part, 12, my_gv >> 1);
+            mbar_arrive_expect_tx(my_full, kVSlotBytes);
+            tma_load_3d(dst, &v_map, 0, page * kPage, (my_gv & 1) * 4, my_full);
             my_gv += kNumVSlots;
+            par ^= 1;
             ++issued;
             have = false;
           }
@@ -606,13 +654,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         }
         if (!ok) {
           if (lane == 0) report_timeout(prm.status);
-          if (issued > 0 && lane < kNumVSlots) mbar_wait(bar(B_VFULL + lane), (issued - 1) & 1);
+          if (issued > 0 && lane < kNumVSlots) mbar_wait(my_full, (issued - 1) & 1);
         }
       }
     } else if (wid == 5) {
       // ---- MMA issuer: O (+)= P~ V_t ; two N = 256 halves, four K = 16 steps each
       if (lane == 0) {
         constexpr uint32_t idesc = make_idesc_bf16(128, 256, false, true);
+        constexpr uint32_t dhi = smem_desc_hi_sw128(1024);
+        const uint32_t vlo0 = smem_desc_lo(smem_base + kOffV, kBoxBytes);
+        const uint32_t plo0 = smem_desc_lo(smem_base + kOffP, 16);
+        uint32_t slot = 0, vpar = 0;
         while (ok && iter.next(u)) {
           for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
             const uint32_t s = gt & 1, k = gt >> 1;
@@ -620,23 +672,24 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             if (!ok) break;
             ok = mbar_wait(bar(B_OREADY + s), k & 1);
             if (!ok) break;
-            const uint32_t pbase = smem_base + kOffP + s * kPStride;
-#pragma unroll
-            for (int nh = 0; nh < 2; ++nh, ++gv) {
-              const uint32_t slot = gv % kNumVSlots, rnd = gv / kNumVSlots;
-              ok = ok && mbar_wait(bar(B_VFULL + slot), rnd & 1);
-              if (ok) {
-                tc_fence_after_sync();
-                if (nh == 0) AMLA_STAMP(prm, part, 15, gt);
-                const uint32_t vbase = smem_base + kOffV + slot * kVSlotBytes;
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                  const uint64_t ad = make_smem_desc_sw128(pbase + kk * 32, 16, 1024);
-                  const uint64_t bd = make_smem_desc_sw128(vbase + kk * 2048, kBoxBytes, 1024);
-                  mma_ss(tbase + nh * 256, ad, bd, idesc, (t > u.t0 || kk > 0) ? 1u : 0u);
-                }
-                mma_commit(bar(B_VEMPTY + slot));
+            const uint32_t plo = plo0 + s * (kPStride >> 4);
+            const uint32_t acc0 = t > u.t0 ? 1u : 0u;
+#pragma unroll 1
+            for (int nh = 0; nh < 2; ++nh) {
+              ok = mbar_wait(bar(B_VFULL) + 8 * slot, vpar);
+              if (!ok) break;
+              tc_fence_after_sync();
+              if (nh == 0) AMLA_STAMP(prm, part, 15, gt);
+              uint32_t vlo = vlo0 + slot * (kVSlotBytes >> 4);
+              uint32_t pl = plo;
+              uint32_t acc = acc0;
+#pragma unroll 1
+              for (int kk = 0; kk < 4; ++kk) {
+                mma_ss(tbase + nh * 256, smem_desc_join(pl, dhi), smem_desc_join(vlo, dhi), idesc, acc);
+                acc = 1; pl += 2; vlo += 128;
               }
+              mma_commit(bar(B_VEMPTY) + 8 * slot);
+              if (++slot == kNumVSlots) { slot = 0; vpar ^= 1; }
             }
             if (!ok) break;
             mma_commit(bar(B_PVDONE + s));
@@ -719,12 +772,15 @@ cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* 
   *unsupported = 0;
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) { *unsupported = 1; return cudaErrorNotSupported; }
+  // K: the cache seen as (64 columns, 8 rows of a group, 9 column blocks, row groups); one box = a page's 64 keys x
+  // 3 column blocks, laid out in shared memory as [row group][column block][8 keys][64 columns], so that a
+  // K-major operand descriptor with a group stride of 3 KB walks the keys of one column block.
   CUtensorMap map;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(kDqk), static_cast<cuuint64_t>(prm.num_blocks) * kPage};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(kDqk) * 2};
-  const cuuint32_t box[2] = {64, 64};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult cr = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(prm.kv), dims, strides,
+  const cuuint64_t dims[4] = {64, 8, static_cast<cuuint64_t>(kDqk / 64), static_cast<cuuint64_t>(prm.num_blocks) * 8};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kDqk) * 2, 128, static_cast<cuuint64_t>(kDqk) * 2 * 8};
+  const cuuint32_t box[4] = {64, 8, 3, 8};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult cr = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(prm.kv), dims, strides,
                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;

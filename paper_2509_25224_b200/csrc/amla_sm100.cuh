@@ -74,12 +74,10 @@ __device__ __forceinline__ bool mbar_probe(uint32_t bar, uint32_t parity) {
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
 
-// Waits for the phase with the given parity to complete; false after kWaitLimitNs.
-template <bool kClusterAcquire = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (int i = 0; i < 64; ++i) {
-    if (kClusterAcquire ? mbar_test_cluster_acquire(bar, parity) : mbar_test(bar, parity)) return true;
-  }
+// Slow path of a wait, kept out of line so that the many call sites stay small (the role loops are
+// executed by single warps and are sensitive to instruction-cache footprint).
+template <bool kClusterAcquire>
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
   const uint64_t t0 = global_timer_ns();
   while (true) {
     for (int i = 0; i < 256; ++i) {
@@ -87,6 +85,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     if (global_timer_ns() - t0 > kWaitLimitNs) return false;
   }
+}
+
+// Waits for the phase with the given parity to complete; false after kWaitLimitNs.
+template <bool kClusterAcquire = false>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (kClusterAcquire ? mbar_test_cluster_acquire(bar, parity) : mbar_test(bar, parity)) return true;
+  return mbar_wait_slow<kClusterAcquire>(bar, parity);
 }
 
 // ------------------------------------------------------------------ fences
@@ -148,6 +153,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const void* tmap,
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+// 4-D tiled load.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tmap, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
 // Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the bytes are
@@ -234,6 +246,18 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
   d |= static_cast<uint64_t>(1) << 46;
   d |= static_cast<uint64_t>(2) << 61;
   return d;
+}
+
+// The same descriptor split in halves: only the low word depends on the address, so an issue loop can
+// keep the high word and step the low word by (byte offset >> 4).
+__host__ __device__ constexpr uint32_t smem_desc_hi_sw128(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+}
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+  return ((smem_addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t smem_desc_join(uint32_t lo, uint32_t hi) {
+  return (static_cast<uint64_t>(hi) << 32) | lo;
 }
 
 // Instruction descriptor, kind::f16 with bf16 inputs and fp32 accumulation:
