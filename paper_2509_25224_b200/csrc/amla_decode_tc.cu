@@ -32,15 +32,17 @@ using namespace sm100;
 
 namespace {
 
+constexpr int kNumCopyWarps = 4;         // score CTA: warps that move staged P~ to the value CTA
 #ifdef AMLA_TRACE
-constexpr int kThreads = 256;            // trace builds add warp 7, which watches the K slots fill
+constexpr int kThreads = 32 * (7 + kNumCopyWarps);   // trace builds add a last warp, which watches the K slots fill
 #else
-constexpr int kThreads = 224;            // warps 0-3: softmax / correction, 4: TMA, 5: MMA + TMEM alloc, 6: copy / relay
+constexpr int kThreads = 32 * (6 + kNumCopyWarps);   // warps 0-3: softmax / correction, 4: TMA producers, 5: MMA issuer + TMEM alloc, 6..: P copy
 #endif
 constexpr uint32_t kBoxBytes = 64 * 64 * 2;             // one 64-key x 64-column TMA box
 constexpr uint32_t kPBytes = 128 * 64 * 2;              // P~ of one 64-key half: 128 rows x 128 B
 constexpr uint32_t kPXfer = kPBytes + 128 * 4;          // ... followed by the 128 per-row integers
-constexpr uint32_t kPStride = 17 * 1024;                // distance between the two P buffers
+constexpr uint32_t kPStride = 17 * 1024;                // distance between P buffers
+constexpr int kNumP = 4;                                // P buffers in the value CTA (pages the softmax may run ahead)
 
 // ---- score CTA
 constexpr int kNumKSlots = 3;
@@ -48,22 +50,22 @@ constexpr uint32_t kKPageBytes = 3 * kBoxBytes;         // 64 keys x 3 column bl
 constexpr uint32_t kKSlotBytes = 2 * kKPageBytes;       // 128 keys x 192 columns (two pages stacked)
 constexpr uint32_t kKGroupStride = 3 * 1024;            // distance between 8-row groups inside a slot
 constexpr uint32_t kOffQRope = 0;                       // 128 rows x 64 bf16, 128-byte swizzle
-constexpr uint32_t kOffStage = 128 * 64 * 2;            // 2 x kPStride
+constexpr uint32_t kOffStage = 128 * 64 * 2;            // 2 x kPStride: P~ and N of a page, before the copy to the value CTA
 constexpr uint32_t kOffK = kOffStage + 2 * kPStride;
-constexpr uint32_t kOffABars = kOffK + kNumKSlots * kKSlotBytes;
+constexpr uint32_t kEndA = kOffK + kNumKSlots * kKSlotBytes;
 // ---- value CTA
-constexpr int kNumVSlots = 5;
+constexpr int kNumVSlots = 4;
 constexpr uint32_t kVSlotBytes = 4 * kBoxBytes;         // 64 keys x 256 columns
 constexpr uint32_t kOffV = 0;
-constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;    // 2 x kPStride (P~ then N)
-constexpr uint32_t kOffFin = kOffP + 2 * kPStride;      // float2 [2][128] (1/(l*S16), lse)
-constexpr uint32_t kOffBBars = kOffFin + 2 * 128 * 8;
+constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;    // kNumP x kPStride (P~ then N)
+constexpr uint32_t kOffFin = kOffP + kNumP * kPStride;  // float2 [2][128] (1/(l*S16), lse)
+constexpr uint32_t kEndB = kOffFin + 2 * 128 * 8;
+// ---- both: the barriers sit at the same offset, so that one multicast commit can reach the two CTAs
+constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
 constexpr uint32_t kBarBytes = 512;
-constexpr uint32_t kSmemA = kOffABars + kBarBytes;
-constexpr uint32_t kSmemB = kOffBBars + kBarBytes;
-constexpr uint32_t kSmemBytes = kSmemA > kSmemB ? kSmemA : kSmemB;
+constexpr uint32_t kSmemBytes = kOffBars + kBarBytes;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
-static_assert(kOffK % 1024 == 0 && kOffStage % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 // tensor-memory columns
 constexpr uint32_t kTmemCols = 512;
@@ -71,12 +73,13 @@ constexpr uint32_t kQCol = 0;            // score CTA: latent part of Q, 256 col
 constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 columns
 // value CTA: O occupies columns 0..511
 
-// barrier indices, score CTA
-enum { A_KFULL = 0, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2,
-       A_PEMPTY = A_SEMPTY + 2, A_PSTAGED = A_PEMPTY + 2, A_QREADY = A_PSTAGED + 2, A_QFREE, A_NUM };
-// barrier indices, value CTA
-enum { B_VFULL = 0, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + 2,
-       B_PVDONE = B_OREADY + 2, B_FINFULL = B_PVDONE + 2, B_NUM = B_FINFULL + 2 };
+// Barrier indices.  X_PV is shared: in the value CTA it completes when P V of a page has finished (PVDONE), in the
+// score CTA the same arrival (multicast commit) frees the page's P buffer for the softmax (PEMPTY).
+enum { X_PV = 0, X_COMMON = X_PV + kNumP };
+enum { A_KFULL = X_COMMON, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2,
+       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2, A_QFREE, A_NUM };
+enum { B_VFULL = X_COMMON, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP,
+       B_FINFULL = B_OREADY + kNumP, B_NUM = B_FINFULL + 2 };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
 
 struct Unit {
@@ -153,29 +156,27 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     return;
   }
 
-  const uint32_t bars = smem_base + (is_score ? kOffABars : kOffBBars);
+  const uint32_t bars = smem_base + kOffBars;
   auto bar = [&](int i) { return bars + 8u * i; };
   const uint32_t tmem_slot = bars + kBarBytes - 8;
   // addresses of the peer's barriers / buffers (same dynamic-smem base in both CTAs)
-  const uint32_t peerA_bars = map_to_cta(smem_base + kOffABars, 0);
-  const uint32_t peerB_bars = map_to_cta(smem_base + kOffBBars, 1);
+  const uint32_t peerB_bars = map_to_cta(smem_base + kOffBars, 1);
   const uint32_t peerB_base = map_to_cta(smem_base, 1);
 
   if (tid == 0) {
+    for (int i = 0; i < kNumP; ++i) mbar_init(bar(X_PV + i), 1);
     if (is_score) {
       for (int i = 0; i < kNumKSlots; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
       for (int i = 0; i < 2; ++i) {
         mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 128);
-        mbar_init(bar(A_PEMPTY + i), 1); mbar_init(bar(A_PSTAGED + i), 128);
+        mbar_init(bar(A_PSTAGED + i), 128); mbar_init(bar(A_STAGEFREE + i), 2);
       }
       mbar_init(bar(A_QREADY), 128);
       mbar_init(bar(A_QFREE), 1);
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
-      for (int i = 0; i < 2; ++i) {
-        mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 128);
-        mbar_init(bar(B_PVDONE + i), 1); mbar_init(bar(B_FINFULL + i), 128);
-      }
+      for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 128); }
+      for (int i = 0; i < 2; ++i) mbar_init(bar(B_FINFULL + i), 128);
     }
     fence_mbar_init();
     prefetch_tensormap(&kv_map);
@@ -326,13 +327,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                   pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
                 }
               }
-              // stage P~ and N; the copy warp ships them to the value CTA
-              const uint32_t s = gt & 1, k = gt >> 1;
+              // stage P~ and N; the copy warp ships them to the value CTA.  The staging buffer is free again once
+              // the copy that last read it has landed (the value CTA reports that).
+              const uint32_t s2 = gt & 1, k2 = gt >> 1;
               if (tid == 0) AMLA_STAMP(prm, part, 7, gt);
-              ok = warp_wait(bar(A_PEMPTY + s), (k & 1) ^ 1);
+              ok = warp_wait(bar(A_STAGEFREE + s2), (k2 & 1) ^ 1);
               if (!ok) break;
               if (tid == 0) AMLA_STAMP(prm, part, 8, gt);
-              const uint32_t stg = smem_base + kOffStage + s * kPStride;
+              const uint32_t stg = smem_base + kOffStage + s2 * kPStride;
 #pragma unroll
               for (int c = 0; c < 8; ++c)
                 st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
@@ -341,7 +343,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                                                   : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
               st_shared_b32(stg + kPBytes + r * 4, nword);
               fence_proxy_async_smem();
-              mbar_arrive(bar(A_PSTAGED + s));
+              mbar_arrive(bar(A_PSTAGED + s2));
               if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
               ++gt;
             }
@@ -447,16 +449,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
               tc_fence_after_sync();
               AMLA_STAMP(prm, part, 21, gc);
               uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
-              const int n_ts = g < 2 ? 12 : 8;     // the last four steps take the RoPE columns of Q from shared memory
+              const int n_blk = g < 2 ? 3 : 2;     // the last column block takes the RoPE columns of Q from shared memory
 #pragma unroll 1
-              for (int i = 0; i < n_ts; ++i) {
-                mma_ts(d, qa, smem_desc_join(klo, dhi), idesc, acc);
+              for (int cl = 0; cl < n_blk; ++cl) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_ts(d, qa + 8 * kk, smem_desc_join(klo + 2 * kk, dhi), idesc, kk == 0 ? acc : 1u);
                 acc = 1;
-                qa += 8;
-                klo += ((i & 3) == 3) ? 64 - 6 : 2;   // next K step inside the block, or on to the next column block
+                qa += 32;
+                klo += 64;
               }
               if (g == 2) {
-#pragma unroll 1
+#pragma unroll
                 for (int kk = 0; kk < 4; ++kk) mma_ss(d, smem_desc_join(qlo0 + 2 * kk, qhi), smem_desc_join(klo + 2 * kk, dhi), idesc, 1u);
               }
               AMLA_STAMP(prm, part, 26, gc);
@@ -477,7 +480,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         if (!ok) report_timeout(prm.status);
       }
 #ifdef AMLA_TRACE
-    } else if (wid == 7) {
+    } else if (wid == 6 + kNumCopyWarps) {
       // trace builds: lane l watches K slot l and stamps the arrival of its data (non-blocking polls)
       if (prm.trace) {
         Cursor<true> cur(prm, part);
@@ -495,21 +498,43 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         }
       }
 #endif
-    } else if (wid == 6) {
-      // ---- copy issuer: staged P~ / N of one half -> value CTA, counted on its PFULL barrier
-      if (lane == 0) {
+    } else if (wid >= 6 && wid < 6 + kNumCopyWarps) {
+      // ---- copy warps: staged P~ / N of a page -> a free P buffer of the value CTA, by asynchronous remote stores
+      // counted on its PFULL barrier.  (A bulk copy would queue behind the K loads in this SM's copy engine and
+      // arrive thousands of cycles later; remote stores issued by the softmax threads themselves would stall them
+      // at the rate of the SM-to-SM path.)  Warps c and c + 2 serve the pages of parity c -- staging buffer c --
+      // and move one half of the buffer each, so every warp sees every phase of the barriers it waits on.  The
+      // staging buffer is free as soon as both have read their half into registers.
+      {
+        const uint32_t c = (wid - 6) & 1, half = (wid - 6) >> 1;
+        constexpr int kChunks = 17;                         // 512-byte chunks per warp (33 in total)
         while (ok && iter.next(u)) {
           for (int t = u.t0; t < u.t1; ++t, ++gt) {
-            const uint32_t s = gt & 1, k = gt >> 1;
-            ok = mbar_wait(bar(A_PSTAGED + s), k & 1);
+            if ((gt & 1) != c) continue;
+            const uint32_t pb = gt % kNumP;
+            ok = warp_wait(bar(A_PSTAGED + c), (gt >> 1) & 1);
             if (!ok) break;
-            const uint32_t pfull = peerB_bars + 8u * (B_PFULL + s);
-            AMLA_STAMP(prm, part, 23, gt);
-            mbar_arrive_expect_tx_cluster(pfull, kPXfer);
-            bulk_copy_to_cluster(peerB_base + kOffP + s * kPStride, smem_base + kOffStage + s * kPStride, kPXfer, pfull);
+            const uint32_t src = smem_base + kOffStage + c * kPStride + (half * kChunks * 32 + lane) * 16;
+            uint32_t v[kChunks][4];
+#pragma unroll
+            for (int i = 0; i < kChunks; ++i) {
+              if (half * kChunks + i < 33)
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i][0]), "=r"(v[i][1]), "=r"(v[i][2]), "=r"(v[i][3]) : "r"(src + i * 512));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(A_STAGEFREE + c));
+            ok = warp_wait(bar(X_PV + pb), ((gt / kNumP) & 1) ^ 1);      // P V that last read the buffer is done
+            if (!ok) break;
+            const uint32_t pfull = peerB_bars + 8u * (B_PFULL + pb);
+            const uint32_t dst = peerB_base + kOffP + pb * kPStride + (half * kChunks * 32 + lane) * 16;
+            if (lane == 0 && half == 0) { AMLA_STAMP(prm, part, 23, gt); mbar_arrive_expect_tx_cluster(pfull, kPXfer); }
+#pragma unroll
+            for (int i = 0; i < kChunks; ++i) {
+              if (half * kChunks + i < 33) st_async_v4(dst + i * 512, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
+            }
           }
         }
-        if (!ok) report_timeout(prm.status);
+        if (!ok && lane == 0) report_timeout(prm.status);
       }
     }
   } else {
@@ -521,8 +546,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
       while (ok && iter.next(u)) {
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
-          const uint32_t s = gt & 1, k = gt >> 1;
-          ok = warp_wait(bar(B_PFULL + s), k & 1);
+          const uint32_t s = gt % kNumP, k = gt / kNumP;
+          ok = warp_wait<true>(bar(B_PFULL + s), k & 1);
           if (!ok) break;
           if (tid == 0) AMLA_STAMP(prm, part, 13, gt);
           const uint32_t nword = ld_shared_b32(smem_base + kOffP + s * kPStride + kPBytes + r * 4);
@@ -530,7 +555,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           if (__any_sync(0xffffffffu, mine) && t > u.t0) {
             // lines 13-16: O <- AS_FP32(AS_INT32(O) + N), after P V of the previous page has landed
             const uint32_t gp = gt - 1;
-            ok = warp_wait(bar(B_PVDONE + (gp & 1)), (gp >> 1) & 1);
+            ok = warp_wait(bar(X_PV + gp % kNumP), (gp / kNumP) & 1);
             if (!ok) break;
             tc_fence_after_sync();
             // two 32-column chunks in flight: the load of one overlaps the arithmetic of the other
@@ -567,7 +592,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         // ---- epilogue (line 20): out = O / (l * S16)
         {
           const uint32_t gl = gt - 1;
-          ok = warp_wait(bar(B_PVDONE + (gl & 1)), (gl >> 1) & 1);
+          ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
           ok = warp_wait<true>(bar(B_FINFULL + (un & 1)), (un >> 1) & 1);
           if (!ok) break;
@@ -667,11 +692,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         uint32_t slot = 0, vpar = 0;
         while (ok && iter.next(u)) {
           for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
-            const uint32_t s = gt & 1, k = gt >> 1;
-            ok = mbar_wait(bar(B_PFULL + s), k & 1);
+            const uint32_t s = gt % kNumP, k = gt / kNumP;
+            ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
             if (!ok) break;
             ok = mbar_wait(bar(B_OREADY + s), k & 1);
             if (!ok) break;
+            fence_proxy_async_smem();      // P~ was written through the generic proxy (remote asynchronous stores)
             const uint32_t plo = plo0 + s * (kPStride >> 4);
             const uint32_t acc0 = t > u.t0 ? 1u : 0u;
 #pragma unroll 1
@@ -683,33 +709,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
               uint32_t vlo = vlo0 + slot * (kVSlotBytes >> 4);
               uint32_t pl = plo;
               uint32_t acc = acc0;
-#pragma unroll 1
-              for (int kk = 0; kk < 4; ++kk) {
-                mma_ss(tbase + nh * 256, smem_desc_join(pl, dhi), smem_desc_join(vlo, dhi), idesc, acc);
-                acc = 1; pl += 2; vlo += 128;
-              }
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                mma_ss(tbase + nh * 256, smem_desc_join(pl + 2 * kk, dhi), smem_desc_join(vlo + 128 * kk, dhi), idesc, kk == 0 ? acc : 1u);
               mma_commit(bar(B_VEMPTY) + 8 * slot);
               if (++slot == kNumVSlots) { slot = 0; vpar ^= 1; }
             }
             if (!ok) break;
-            mma_commit(bar(B_PVDONE + s));
+            mma_commit_multicast(bar(X_PV + s), 3);   // PVDONE here, PEMPTY in the score CTA
             AMLA_STAMP(prm, part, 16, gt);
           }
           if (!ok) break;
-        }
-        if (!ok) report_timeout(prm.status);
-      }
-    } else if (wid == 6) {
-      // ---- relay: tell the score CTA that a P buffer is free once its P V has completed
-      if (lane == 0) {
-        while (ok && iter.next(u)) {
-          for (int t = u.t0; t < u.t1; ++t, ++gt) {
-            const uint32_t s = gt & 1, k = gt >> 1;
-            ok = mbar_wait(bar(B_PVDONE + s), k & 1);
-            if (!ok) break;
-            AMLA_STAMP(prm, part, 17, gt);
-            mbar_arrive_cluster(peerA_bars + 8u * (A_PEMPTY + s));
-          }
         }
         if (!ok) report_timeout(prm.status);
       }

@@ -292,6 +292,25 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Like mma_commit, but the arrival is delivered to the barrier at the same shared-memory offset in every
+// CTA of the cluster named in cta_mask (bit i = CTA rank i).
+__device__ __forceinline__ void mma_commit_multicast(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(cta_mask) : "memory");
+}
+
+// Asynchronous stores into the shared memory of a CTA of the cluster; each adds its size to the transaction
+// count of a barrier of that CTA.  Generic-proxy writes: a consumer that reads them through the async proxy
+// (TMA, tcgen05.mma) fences with fence.proxy.async after its wait.
+__device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void st_async_b32(uint32_t cluster_addr, uint32_t a, uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+               ::"r"(cluster_addr), "r"(a), "r"(cluster_bar) : "memory");
+}
+
 // Byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled tile whose rows are 128 B
 // (the pattern TMA's SWIZZLE_128B produces and the descriptors above expect; the tile base must be
 // 1024-byte aligned): chunk index XOR (row mod 8).
