@@ -59,7 +59,8 @@ constexpr uint32_t kVSlotBytes = 4 * kBoxBytes;         // 64 keys x 256 columns
 constexpr uint32_t kOffV = 0;
 constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;    // kNumP x kPStride (P~ then N)
 constexpr uint32_t kOffFin = kOffP + kNumP * kPStride;  // float2 [2][128] (1/(l*S16), lse)
-constexpr uint32_t kEndB = kOffFin + 2 * 128 * 8;
+constexpr uint32_t kOffEpi = kOffFin + 2 * 128 * 8;     // epilogue transpose tiles: 4 warps x 32 rows x 128 B
+constexpr uint32_t kEndB = kOffEpi + 4 * 32 * 128;
 // ---- both: the barriers sit at the same offset, so that one multicast commit can reach the two CTAs
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
 constexpr uint32_t kBarBytes = 512;
@@ -140,6 +141,33 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
   return __all_sync(0xffffffffu, mbar_wait<kClusterAcquire>(bar, parity));
 }
 
+// Brings the nine 128-byte lines of one query row of a unit into L2 ahead of the loads that move it on chip.
+__device__ __forceinline__ void prefetch_q_row(const DecodeParams& prm, const Unit& u, int row) {
+  if (row < u.nrows) {
+    const char* p = reinterpret_cast<const char*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + row) * kDqk);
+#pragma unroll
+    for (int i = 0; i < 9; ++i) prefetch_l2(p + 128 * i);
+  }
+}
+
+// One query row: four 64-column blocks [blk0, blk0 + 4) of its latent part go from global memory into the
+// 128 tensor-memory columns that hold them (two bf16 per column), two blocks (16 loads) at a time.
+__device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int blk0, uint32_t taddr) {
+#pragma unroll 1
+  for (int b = blk0; b < blk0 + 4; b += 2) {
+    uint32_t x0[32], x1[32];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint4 v = valid ? __ldg(qrow + b * 8 + c) : make_uint4(0, 0, 0, 0);
+      x0[4 * c] = v.x; x0[4 * c + 1] = v.y; x0[4 * c + 2] = v.z; x0[4 * c + 3] = v.w;
+      const uint4 w = valid ? __ldg(qrow + b * 8 + 8 + c) : make_uint4(0, 0, 0, 0);
+      x1[4 * c] = w.x; x1[4 * c + 1] = w.y; x1[4 * c + 2] = w.z; x1[4 * c + 3] = w.w;
+    }
+    tmem_st_32x32b_x32(taddr + b * 32, x0);
+    tmem_st_32x32b_x32(taddr + b * 32 + 32, x1);
+  }
+}
+
 }  // namespace
 
 template <int kMode, bool kGuard>
@@ -154,6 +182,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   if (smem_base & 1023u) {   // the swizzled tiles assume a 1024-byte aligned window; identical in both CTAs
     if (tid == 0) report_timeout(prm.status);
     return;
+  }
+
+  if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
+    UnitIter first(prm, part);
+    Unit fu;
+    if (first.next(fu)) prefetch_q_row(prm, fu, tid);
   }
 
   const uint32_t bars = smem_base + kOffBars;
@@ -171,7 +205,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 128);
         mbar_init(bar(A_PSTAGED + i), 128); mbar_init(bar(A_STAGEFREE + i), 2);
       }
-      mbar_init(bar(A_QREADY), 128);
+      mbar_init(bar(A_QREADY), 256);
       mbar_init(bar(A_QFREE), 1);
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
@@ -214,28 +248,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         tc_fence_after_sync();
         if (tid == 0) AMLA_STAMP(prm, part, 10, un);
         {
+          // this warpgroup brings in the first 256 latent columns of its rows; the copy warps, idle at this
+          // point, bring in the other 256 and the RoPE columns
           const bool valid = r < u.nrows;
           const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDqk);
-#pragma unroll 1
-          for (int blk = 0; blk < 8; blk += 2) {
-            uint32_t r0[32], r1[32];
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              const uint4 v = valid ? __ldg(qrow + blk * 8 + c) : make_uint4(0, 0, 0, 0);
-              r0[4 * c] = v.x; r0[4 * c + 1] = v.y; r0[4 * c + 2] = v.z; r0[4 * c + 3] = v.w;
-              const uint4 w = valid ? __ldg(qrow + blk * 8 + 8 + c) : make_uint4(0, 0, 0, 0);
-              r1[4 * c] = w.x; r1[4 * c + 1] = w.y; r1[4 * c + 2] = w.z; r1[4 * c + 3] = w.w;
-            }
-            tmem_st_32x32b_x32(tbase + lane_base + kQCol + blk * 32, r0);
-            tmem_st_32x32b_x32(tbase + lane_base + kQCol + blk * 32 + 32, r1);
-          }
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 v = valid ? __ldg(qrow + 64 + c) : make_uint4(0, 0, 0, 0);
-            st_shared_v4(smem_base + kOffQRope + sw128_offset(r, c), v.x, v.y, v.z, v.w);
-          }
+          load_q_latent(qrow, valid, 0, tbase + lane_base + kQCol);
           tmem_wait_st();
-          fence_proxy_async_smem();
         }
         tc_fence_before_sync();
         mbar_arrive(bar(A_QREADY));
@@ -508,7 +526,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       {
         const uint32_t c = (wid - 6) & 1, half = (wid - 6) >> 1;
         constexpr int kChunks = 17;                         // 512-byte chunks per warp (33 in total)
+        const int qr = (wid & 3) * 32 + lane;               // query row whose second half this thread loads
+        const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
         while (ok && iter.next(u)) {
+          {
+            ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool valid = qr < u.nrows;
+            const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? qr : 0)) * kDqk);
+            load_q_latent(qrow, valid, 4, tbase + q_lane_base + kQCol);
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+              const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
+              st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
+            }
+            tmem_wait_st();
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(bar(A_QREADY));
+            ++un;
+            UnitIter peek = iter;              // the next unit's Q goes to L2 while this one is computed
+            Unit nu;
+            if (peek.next(nu)) prefetch_q_row(prm, nu, qr);
+          }
           for (int t = u.t0; t < u.t1; ++t, ++gt) {
             if ((gt & 1) != c) continue;
             const uint32_t pb = gt % kNumP;
@@ -605,30 +646,55 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             inv = __uint_as_float(x); lse = __uint_as_float(y);
           }
           const bool valid = r < u.nrows;
-          __nv_bfloat16* orow = prm.out + (static_cast<size_t>(u.b) * prm.R + u.r0 + r) * kDv;
-          float* prow = prm.part_o + (static_cast<size_t>(u.slot < 0 ? 0 : u.slot) * kRowBlock + r) * kDv;
+          // 32 columns at a time: each lane scales its row, the warp transposes the 32 x 32 tile through shared
+          // memory (16-byte units XOR-swizzled by row), and writes whole 128-byte (FP32 partial) or 64-byte (bf16)
+          // row pieces, so that a store instruction covers full lines instead of 32 scattered sectors.
+          const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
+          const int rows_here = min(32, u.nrows - wid * 32);          // valid rows of this warp's 32 (may be <= 0)
+          __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + u.r0 + wid * 32) * kDv;
+          float* pbase = prm.part_o + (static_cast<size_t>(u.slot < 0 ? 0 : u.slot) * kRowBlock + wid * 32) * kDv;
+          uint32_t o[2][32];
+          tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
 #pragma unroll 1
-          for (int c = 0; c < 16; ++c) {
-            uint32_t o[32];
-            tmem_ld_32x32b_x32(tbase + lane_base + 32 * c, o);
-            tmem_wait_ld();
-            if (valid) {
+          for (int c = 0; c < 16; c += 2) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              tmem_wait_ld();
+              if (c + e + 1 < 16) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (c + e + 1), o[e ^ 1]);
+              const int cc = c + e;
+              __syncwarp();                                           // the tile is free again (previous read-back done)
               if (u.slot < 0) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int j = 0; j < 4; ++j) {
+                  const uint32_t w0 = pack_bf16x2(__uint_as_float(o[e][8 * j + 0]) * inv, __uint_as_float(o[e][8 * j + 1]) * inv);
+                  const uint32_t w1 = pack_bf16x2(__uint_as_float(o[e][8 * j + 2]) * inv, __uint_as_float(o[e][8 * j + 3]) * inv);
+                  const uint32_t w2 = pack_bf16x2(__uint_as_float(o[e][8 * j + 4]) * inv, __uint_as_float(o[e][8 * j + 5]) * inv);
+                  const uint32_t w3 = pack_bf16x2(__uint_as_float(o[e][8 * j + 6]) * inv, __uint_as_float(o[e][8 * j + 7]) * inv);
+                  st_shared_v4(epi + lane * 128 + ((j ^ (lane & 7)) << 4), w0, w1, w2, w3);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {                         // 8 rows x 64 B per instruction
+                  const int row = 8 * k + (lane >> 2), j = lane & 3;
                   uint4 v;
-                  v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-                  v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-                  v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-                  v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-                  *reinterpret_cast<uint4*>(orow + 32 * c + 8 * i) = v;
+                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                               : "r"(epi + row * 128 + ((j ^ (row & 7)) << 4)));
+                  if (row < rows_here) *reinterpret_cast<uint4*>(obase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * j) = v;
                 }
               } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  float4 v = make_float4(__uint_as_float(o[4 * i + 0]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
-                                         __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv);
-                  *reinterpret_cast<float4*>(prow + 32 * c + 4 * i) = v;
+                for (int j = 0; j < 8; ++j)
+                  st_shared_v4(epi + lane * 128 + ((j ^ (lane & 7)) << 4),
+                               __float_as_uint(__uint_as_float(o[e][4 * j + 0]) * inv), __float_as_uint(__uint_as_float(o[e][4 * j + 1]) * inv),
+                               __float_as_uint(__uint_as_float(o[e][4 * j + 2]) * inv), __float_as_uint(__uint_as_float(o[e][4 * j + 3]) * inv));
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {                         // 4 rows x 128 B per instruction
+                  const int row = 4 * k + (lane >> 3), j = lane & 7;
+                  uint4 v;
+                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                               : "r"(epi + row * 128 + ((j ^ (row & 7)) << 4)));
+                  if (row < rows_here) *reinterpret_cast<uint4*>(pbase + static_cast<size_t>(row) * kDv + 32 * cc + 4 * j) = v;
                 }
               }
             }
