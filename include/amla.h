@@ -28,7 +28,8 @@ typedef enum {
   AMLA_ERR_UNSUPPORTED = -2,    /* shape or device outside what the kernels cover       */
   AMLA_ERR_WORKSPACE = -3,      /* workspace smaller than amla_mla_decode_workspace_size */
   AMLA_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed                    */
-  AMLA_ERR_DEVICE_TIMEOUT = -5  /* a bounded device-side wait ran out (see amla_check_status) */
+  AMLA_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait ran out (see amla_check_status) */
+  AMLA_ERR_STATIC_LIMIT = -6    /* amla_mla_decode_static: problem or device beyond its built-in scratch */
 } amla_status;
 
 /* Rescale variants, for A/B measurements (flags argument of amla_mla_decode_ex).
@@ -98,7 +99,35 @@ int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_ta
                     int max_blocks_per_seq, void* out, float* lse, void* workspace,
                     size_t workspace_bytes, void* cuda_stream);
 
-/* Same, with a flags word selecting a rescale variant (see the enum above). */
+/*
+ * amla_mla_decode without a workspace argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a serving loop that must never enter the
+ * allocator on its hot path, a process whose device memory was carved up completely at start-up, a plugin that
+ * is handed input and output buffers and nothing else.  The scratch the decode needs (schedule prefix, status
+ * word, FP32 partials of split sequences) lives in a fixed array inside the library image instead: about 37 MiB
+ * that every GPU which loads the library holds until the process exits.  The call itself performs no cudaMalloc,
+ * cudaFree or any other allocating call.
+ *
+ * Arguments, layouts, the visibility rule and the results are those of amla_mla_decode (default rescale variant).
+ * Limits: B * ceil(Sq*H/128) <= AMLA_STATIC_MAX_ITEMS and a device with at most AMLA_STATIC_MAX_SMS SMs; beyond
+ * either the call returns AMLA_ERR_STATIC_LIMIT and launches nothing.
+ *
+ * The first call on a device looks up the device address of the array (a one-time query, made with that device
+ * current); make that first call before any stream capture begins.  All calls on a device share the one array and
+ * it keeps the previous call's contents: that is harmless, because each call rewrites everything it later reads,
+ * but two calls whose kernels overlap on the GPU (different streams, no ordering between them) race on it and
+ * give undefined results.  Order such calls, or use amla_mla_decode with one workspace per stream.
+ * The bounded-wait status word is inside the array; amla_check_status does not apply to this entry point.
+ */
+#define AMLA_STATIC_MAX_ITEMS 4096
+#define AMLA_STATIC_MAX_SMS 148
+int amla_mla_decode_static(const void* q, const void* kv_cache, const int32_t* block_table,
+                           const int32_t* seqlens, float softmax_scale, int B, int Sq, int H, int num_blocks,
+                           int max_blocks_per_seq, void* out, float* lse, void* cuda_stream);
+
+/* Same as amla_mla_decode, with a flags word selecting a rescale variant (see the enum above). */
 int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block_table,
                        const int32_t* seqlens, float softmax_scale, int B, int Sq, int H,
                        int num_blocks, int max_blocks_per_seq, void* out, float* lse, void* workspace,

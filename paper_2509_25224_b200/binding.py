@@ -35,7 +35,7 @@ DEFAULT_FLAGS = RESCALE_ALG2 | lazy(DEFAULT_TAU)   # what amla_mla_decode (witho
 EXPORTS = [
     "amla_status_string", "amla_mla_decode_workspace_size", "amla_mla_decode", "amla_mla_decode_ex",
     "amla_check_status", "amla_last_launch_count", "amla_plan_host", "amla_profile_enable",
-    "amla_profile_last_ms",
+    "amla_profile_last_ms", "amla_mla_decode_static",
 ]
 
 _lib = None
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.amla_mla_decode.restype = i32
         L.amla_mla_decode_ex.argtypes = dec + [i32]
         L.amla_mla_decode_ex.restype = i32
+        L.amla_mla_decode_static.argtypes = [vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.amla_mla_decode_static.restype = i32
         L.amla_check_status.argtypes = [vp, vp]
         L.amla_check_status.restype = i32
         L.amla_last_launch_count.argtypes = []
@@ -118,6 +120,22 @@ def mla_decode_raw(q_ptr: int, kv_ptr: int, bt_ptr: int, sl_ptr: int, scale: flo
                                       max_blocks_per_seq, out_ptr, lse_ptr, ws_ptr, ws_bytes, stream, int(flags))
     if rc != AMLA_OK:
         raise AmlaError(rc, "amla_mla_decode")
+
+
+def mla_decode_static(q, kv_cache, block_table, seqlens, softmax_scale: float, out, lse) -> None:
+    """amla_mla_decode_static on device tensors: the decode call that takes no workspace and allocates nothing
+    (its scratch is a fixed array inside the library).  `out` and `lse` must be given -- this wrapper allocates
+    nothing either.  Raises AmlaError(-6) when the problem exceeds the built-in scratch."""
+    import torch
+
+    B, Sq, H, _ = q.shape
+    stream = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        rc = lib().amla_mla_decode_static(q.data_ptr(), kv_cache.data_ptr(), block_table.data_ptr(), seqlens.data_ptr(),
+                                          float(softmax_scale), B, Sq, H, kv_cache.shape[0], block_table.shape[1],
+                                          out.data_ptr(), lse.data_ptr(), stream)
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_mla_decode_static")
 
 
 def last_launch_count() -> int:

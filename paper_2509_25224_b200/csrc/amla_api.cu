@@ -93,6 +93,7 @@ extern "C" const char* amla_status_string(int status) {
     case AMLA_ERR_WORKSPACE: return "workspace too small";
     case AMLA_ERR_CUDA: return "CUDA call failed";
     case AMLA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case AMLA_ERR_STATIC_LIMIT: return "problem or device exceeds the built-in scratch of amla_mla_decode_static";
     default: return "unknown status";
   }
 }
