@@ -86,6 +86,17 @@ class ClockSampler:
                 "power_w_max": max(power), "samples": len(sm)}
 
 
+def kernel_source_hash():
+    """sha256 over the CUDA sources of the library (what the ncu counters in profiles/ were taken with)."""
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    for p in sorted(glob.glob(os.path.join(ROOT, "paper_2509_25224_b200", "csrc", "*.cu*"))):
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -269,11 +280,13 @@ def run_gpu(args):
             "kernel_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9,
             "algorithmic_bytes": alg_bytes, "flops": flops,
         })
+        # DRAM bytes per launch from the committed ncu capture; only valid for the kernel sources it was taken with
         traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(traffic_file):
             with open(traffic_file) as f:
                 tr = json.load(f)
-            roof["traffic"] = tr.get(w.name)
+            if tr.get("source_sha256") == kernel_source_hash():
+                roof["traffic"] = tr.get(w.name)
         n_rows = {"tiny": 16, "dsv3": 4096, "mtp": 2048, "stress": 1024, "long": 256}[w.name]
         tf, dt, cores, sample = time_oracle(w, n_rows)
         line = {
