@@ -184,12 +184,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     return;
   }
 
-  if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
-    UnitIter first(prm, part);
-    Unit fu;
-    if (first.next(fu)) prefetch_q_row(prm, fu, tid);
-  }
-
   const uint32_t bars = smem_base + kOffBars;
   auto bar = [&](int i) { return bars + 8u * i; };
   const uint32_t tmem_slot = bars + kBarBytes - 8;
@@ -224,6 +218,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   tc_fence_after_sync();
   const uint32_t tbase = ld_shared_b32(tmem_slot);
   if (tid == 0) AMLA_STAMP(prm, part, is_score ? 0 : 1, 0);
+
+  // Launched with programmatic stream serialization: everything above ran while the schedule kernel was still
+  // going; its prefix array (and the caller's earlier work on the stream) is visible after this wait.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;");
+  if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
+    UnitIter first(prm, part);
+    Unit fu;
+    if (first.next(fu)) prefetch_q_row(prm, fu, tid);
+  }
+
 
   bool ok = true;
   UnitIter iter(prm, part);
@@ -835,8 +840,17 @@ cudaError_t launch_variant(const CUtensorMap& map, const CUtensorMap& vmap, cons
     if (err != cudaSuccess) return err;
     done.fetch_or(bit, std::memory_order_release);
   }
-  kern<<<2 * prm.P, kThreads, kSmemBytes, stream>>>(map, vmap, prm);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * prm.P);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, map, vmap, prm);
 }
 
 }  // namespace

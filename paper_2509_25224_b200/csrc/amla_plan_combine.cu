@@ -12,6 +12,7 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
                             int* __restrict__ prefix, int* __restrict__ status) {
   __shared__ int warp_sums[32];
   __shared__ int carry;
+  asm volatile("griddepcontrol.launch_dependents;");   // the decode kernel may start its set-up; it waits before reading
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   if (tid == 0) { carry = 0; *status = kStatusOk; }
   __syncthreads();
@@ -52,6 +53,7 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
 // and are skipped; items without tiles get out = 0, lse = -inf; split items are merged:
 //   lse = ln sum_s exp(lse_s),  out = sum_s exp(lse_s - lse) * out_s.
 __global__ void combine_kernel(DecodeParams prm) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // launched early (programmatic dependent launch): the partials must be complete
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row_global = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
@@ -75,11 +77,14 @@ __global__ void combine_kernel(DecodeParams prm) {
     if (lane == 0) *lrow = -INFINITY;
     return;
   }
+  // lse of the splits: one split per lane (in rounds of 32), so that the loads overlap
   float mx = -INFINITY;
-  for (int p = p_first; p <= p_last; ++p) {
-    const int slot = plan.slot_of(p, it, p_first);
-    mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(slot) * kRowBlock + rr]);
+  for (int base = 0; base < nsplit; base += 32) {
+    const int sidx = base + lane;
+    if (sidx < nsplit) mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(plan.slot_of(p_first + sidx, it, p_first)) * kRowBlock + rr]);
   }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   if (mx == -INFINITY) {   // no split saw a visible key for this row
     for (int c = lane * 8; c < kDv; c += 32 * 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
     if (lane == 0) *lrow = -INFINITY;
@@ -89,17 +94,27 @@ __global__ void combine_kernel(DecodeParams prm) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) acc[i] = 0.f;
   float tot = 0.f;
-  for (int p = p_first; p <= p_last; ++p) {
-    const int slot = plan.slot_of(p, it, p_first);
-    const float ls = prm.part_lse[static_cast<size_t>(slot) * kRowBlock + rr];
-    const float w = expf(ls - mx);   // 0 for a split that saw nothing (lse_s = -inf)
-    tot += w;
-    const float* src = prm.part_o + (static_cast<size_t>(slot) * kRowBlock + rr) * kDv;
+  for (int base = 0; base < nsplit; base += 32) {
+    const int sidx = base + lane;
+    int my_slot = 0;
+    float my_w = 0.f;
+    if (sidx < nsplit) {
+      my_slot = plan.slot_of(p_first + sidx, it, p_first);
+      my_w = expf(prm.part_lse[static_cast<size_t>(my_slot) * kRowBlock + rr] - mx);   // 0 for a split that saw nothing
+    }
+    const int n_here = min(32, nsplit - base);
+#pragma unroll 2
+    for (int j = 0; j < n_here; ++j) {
+      const float w = __shfl_sync(0xffffffffu, my_w, j);
+      const int slot = __shfl_sync(0xffffffffu, my_slot, j);
+      tot += w;
+      const float* src = prm.part_o + (static_cast<size_t>(slot) * kRowBlock + rr) * kDv;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float4 v = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
-      acc[4 * i + 0] += w * v.x; acc[4 * i + 1] += w * v.y;
-      acc[4 * i + 2] += w * v.z; acc[4 * i + 3] += w * v.w;
+      for (int i = 0; i < 4; ++i) {
+        const float4 v = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
+        acc[4 * i + 0] += w * v.x; acc[4 * i + 1] += w * v.y;
+        acc[4 * i + 2] += w * v.z; acc[4 * i + 3] += w * v.w;
+      }
     }
   }
   const float inv = 1.f / tot;
@@ -124,8 +139,18 @@ cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream) {
   const int warps_per_block = 8;
   const long rows = static_cast<long>(prm.B) * prm.nrb * kRowBlock;
   const int blocks = static_cast<int>((rows + warps_per_block - 1) / warps_per_block);
-  combine_kernel<<<blocks, warps_per_block * 32, 0, stream>>>(prm);
-  return cudaGetLastError();
+  // programmatic dependent launch: the blocks may be placed while the decode kernel drains; they wait inside
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(warps_per_block * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, combine_kernel, prm);
 }
 
 }  // namespace amla
