@@ -45,13 +45,13 @@ constexpr uint32_t kPStride = 17 * 1024;                // distance between P bu
 constexpr int kNumP = 4;                                // P buffers in the value CTA (pages the softmax may run ahead)
 
 // ---- score CTA
-constexpr int kNumKSlots = 3;
+constexpr int kNumKSlots = 4;                           // 192 KB in flight: what the load latency needs at the MMA's rate
 constexpr uint32_t kKPageBytes = 3 * kBoxBytes;         // 64 keys x 3 column blocks: [8 row groups][3 blocks][8 rows][128 B]
 constexpr uint32_t kKSlotBytes = 2 * kKPageBytes;       // 128 keys x 192 columns (two pages stacked)
 constexpr uint32_t kKGroupStride = 3 * 1024;            // distance between 8-row groups inside a slot
 constexpr uint32_t kOffQRope = 0;                       // 128 rows x 64 bf16, 128-byte swizzle
-constexpr uint32_t kOffStage = 128 * 64 * 2;            // 2 x kPStride: P~ and N of a page, before the copy to the value CTA
-constexpr uint32_t kOffK = kOffStage + 2 * kPStride;
+constexpr uint32_t kOffStage = 128 * 64 * 2;            // kPStride: P~ and N of a page, before the copy warps move them to the value CTA
+constexpr uint32_t kOffK = kOffStage + kPStride;
 constexpr uint32_t kEndA = kOffK + kNumKSlots * kKSlotBytes;
 // ---- value CTA
 constexpr int kNumVSlots = 4;
@@ -350,14 +350,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                   pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
                 }
               }
-              // stage P~ and N; the copy warp ships them to the value CTA.  The staging buffer is free again once
-              // the copy that last read it has landed (the value CTA reports that).
-              const uint32_t s2 = gt & 1, k2 = gt >> 1;
+              // stage P~ and N; the copy warps ship them to the value CTA
+              const uint32_t s2 = gt & 1;
               if (tid == 0) AMLA_STAMP(prm, part, 7, gt);
-              ok = warp_wait(bar(A_STAGEFREE + s2), (k2 & 1) ^ 1);
+              // one staging buffer: the copy warps of the previous page must have read it into registers
+              if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
               if (!ok) break;
               if (tid == 0) AMLA_STAMP(prm, part, 8, gt);
-              const uint32_t stg = smem_base + kOffStage + s2 * kPStride;
+              const uint32_t stg = smem_base + kOffStage;
 #pragma unroll
               for (int c = 0; c < 8; ++c)
                 st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
@@ -560,7 +560,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             const uint32_t pb = gt % kNumP;
             ok = warp_wait(bar(A_PSTAGED + c), (gt >> 1) & 1);
             if (!ok) break;
-            const uint32_t src = smem_base + kOffStage + c * kPStride + (half * kChunks * 32 + lane) * 16;
+            const uint32_t src = smem_base + kOffStage + (half * kChunks * 32 + lane) * 16;
             uint32_t v[kChunks][4];
 #pragma unroll
             for (int i = 0; i < kChunks; ++i) {
