@@ -151,17 +151,21 @@ __device__ __forceinline__ void prefetch_q_row(const DecodeParams& prm, const Un
 }
 
 // One query row: four 64-column blocks [blk0, blk0 + 4) of its latent part go from global memory into the
-// 128 tensor-memory columns that hold them (two bf16 per column), two blocks (16 loads) at a time.
+// 128 tensor-memory columns that hold them (two bf16 per column), two blocks at a time.  Every lane reads its own
+// row, so an instruction touches 32 lines; 256-bit loads halve the number of such instructions.
 __device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int blk0, uint32_t taddr) {
 #pragma unroll 1
   for (int b = blk0; b < blk0 + 4; b += 2) {
     uint32_t x0[32], x1[32];
+    if (valid) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 v = valid ? __ldg(qrow + b * 8 + c) : make_uint4(0, 0, 0, 0);
-      x0[4 * c] = v.x; x0[4 * c + 1] = v.y; x0[4 * c + 2] = v.z; x0[4 * c + 3] = v.w;
-      const uint4 w = valid ? __ldg(qrow + b * 8 + 8 + c) : make_uint4(0, 0, 0, 0);
-      x1[4 * c] = w.x; x1[4 * c + 1] = w.y; x1[4 * c + 2] = w.z; x1[4 * c + 3] = w.w;
+      for (int c = 0; c < 4; ++c) {
+        ldg_256(qrow + b * 8 + 2 * c, x0, 8 * c);
+        ldg_256(qrow + b * 8 + 8 + 2 * c, x1, 8 * c);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) { x0[i] = 0; x1[i] = 0; }
     }
     tmem_st_32x32b_x32(taddr + b * 32, x0);
     tmem_st_32x32b_x32(taddr + b * 32 + 32, x1);

@@ -176,6 +176,12 @@ __device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int x, int 
   asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
                ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y) : "memory");
 }
+// 256-bit read-only global load (32-byte aligned address).
+__device__ __forceinline__ void ldg_256(const void* p, uint32_t (&r)[32], int at) {
+  asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[at]), "=r"(r[at + 1]), "=r"(r[at + 2]), "=r"(r[at + 3]), "=r"(r[at + 4]), "=r"(r[at + 5]), "=r"(r[at + 6]), "=r"(r[at + 7])
+               : "l"(p));
+}
 __device__ __forceinline__ void prefetch_l2(const void* p) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
