@@ -471,9 +471,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
 #pragma unroll 1
             for (int g = 0; g < 3; ++g) {
               AMLA_STAMP(prm, part, 25, gc);
-              ok = mbar_wait(bar(A_KFULL) + 8 * slot, kpar);
+              ok = mbar_wait(bar(A_KFULL) + 8 * slot, kpar);    // TMA data -> MMA operand: both async proxy, no fence needed
               if (!ok) break;
-              tc_fence_after_sync();
               AMLA_STAMP(prm, part, 21, gc);
               uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
               const int n_blk = g < 2 ? 3 : 2;     // the last column block takes the RoPE columns of Q from shared memory
@@ -772,6 +771,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             if (!ok) break;
             ok = mbar_wait(bar(B_OREADY + s), k & 1);
             if (!ok) break;
+            tc_fence_after_sync();         // the correction warps may have rewritten O (tcgen05.st) before arriving
             fence_proxy_async_smem();      // P~ was written through the generic proxy (remote asynchronous stores)
             const uint32_t plo = plo0 + s * (kPStride >> 4);
             const uint32_t acc0 = t > u.t0 ? 1u : 0u;
@@ -779,7 +779,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             for (int nh = 0; nh < 2; ++nh) {
               ok = mbar_wait(bar(B_VFULL) + 8 * slot, vpar);
               if (!ok) break;
-              tc_fence_after_sync();
               if (nh == 0) AMLA_STAMP(prm, part, 15, gt);
               uint32_t vlo = vlo0 + slot * (kVSlotBytes >> 4);
               uint32_t pl = plo;
