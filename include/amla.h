@@ -153,7 +153,8 @@ int amla_profile_last_ms(float* ms3);
 /*
  * Host mirror of the device-side split-KV schedule (the plan is not in the paper; it exists because
  * B * ceil(Sq*H/128) work items are far fewer than the SMs).  Items are (sequence, 128-row block)
- * pairs in order; their 64-key tiles form one linear range that is cut into num_parts equal parts.
+ * pairs in order; their 64-key tiles, each non-empty item preceded by 10 overhead positions that stand
+ * for the cost of starting an item, form one linear range that is cut into num_parts equal parts.
  * For every (part, item) intersection ("unit") one record of 6 int32 is written:
  *   part, item, tile_begin, tile_end (within the item), slot (-1 = writes out/lse directly,
  *   otherwise index of its fp32 partial), n_split of the item.

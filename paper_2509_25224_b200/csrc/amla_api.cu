@@ -247,7 +247,8 @@ extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int 
     prefix[it] = acc;
     int n = seqlens[it / nrb];
     if (n < 0) n = 0;
-    acc += (n + kPage - 1) / kPage;
+    const int tiles = (n + kPage - 1) / kPage;
+    acc += tiles > 0 ? tiles + kUnitOverheadTiles : 0;
   }
   prefix[n_items] = acc;
   const Plan plan = Plan::make(prefix, n_items, num_parts);
@@ -259,9 +260,11 @@ extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int 
       int g = g0;
       while (g < g1) {
         const int it = plan.item_of_tile(g);
-        const int a = prefix[it], e = prefix[it + 1];
-        const int t0 = g - a, t1 = (e < g1 ? e : g1) - a;
-        g = a + t1;
+        const int a = plan.first_tile(it), e = prefix[it + 1];
+        const int lo = g > a ? g : a, hi = e < g1 ? e : g1;
+        g = e < g1 ? e : g1;
+        if (hi <= lo) continue;
+        const int t0 = lo - a, t1 = hi - a;
         int p_first, p_last;
         const int nsplit = plan.item_parts(it, &p_first, &p_last);
         if (n_units < max_units) {

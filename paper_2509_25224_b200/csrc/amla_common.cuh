@@ -59,16 +59,22 @@ constexpr int kTraceTiles = 96;
 
 // ---------------------------------------------------------------------------------------------
 // Split-KV schedule.  Items (sequence b, row block rb) in order it = b * nrb + rb own
-// ceil(N_b / 64) tiles each; prefix[it] is the linear index of an item's first tile and
-// L = prefix[n_items] the total.  Part p owns linear tiles [p*L/P, (p+1)*L/P).
+// ceil(N_b / 64) tiles each.  Starting an item costs a cluster a fixed amount of time (its Q rows,
+// the pipeline fill, the epilogue) that is worth about kUnitOverheadTiles tiles, so the schedule
+// balances a linear range in which every non-empty item is preceded by that many overhead
+// positions: prefix[it] is the position where item `it` begins (overhead first, then its tiles),
+// L = prefix[n_items] the total, and part p owns positions [p*L/P, (p+1)*L/P).  A part does the
+// tiles whose positions it owns; overhead positions carry no work.
 // ---------------------------------------------------------------------------------------------
+constexpr int kUnitOverheadTiles = 10;
+
 struct Plan {
   const int* prefix;
   int n_items;
   int L;
   int P;
 
-  // With fewer tiles than parts only the first L parts get work (one tile each).
+  // With fewer positions than parts only the first L parts exist (one position each).
   __host__ __device__ static Plan make(const int* prefix, int n_items, int max_parts) {
     Plan pl;
     pl.prefix = prefix;
@@ -97,10 +103,13 @@ struct Plan {
     }
     return lo;
   }
-  // Parts [p_first, p_last] that touch item `it`; returns the split count (0 for an empty item).
+  // Position of the first tile of a non-empty item.
+  __host__ __device__ int first_tile(int it) const { return prefix[it] + kUnitOverheadTiles; }
+  // Parts [p_first, p_last] that hold tiles of item `it`; returns the split count (0 for an empty item).
   __host__ __device__ int item_parts(int it, int* p_first, int* p_last) const {
-    const int a = prefix[it], e = prefix[it + 1];
-    if (e <= a) { *p_first = 0; *p_last = -1; return 0; }
+    const int e = prefix[it + 1];
+    if (e <= prefix[it]) { *p_first = 0; *p_last = -1; return 0; }
+    const int a = first_tile(it);
     *p_first = part_of_tile(a);
     *p_last = part_of_tile(e - 1);
     return *p_last - *p_first + 1;

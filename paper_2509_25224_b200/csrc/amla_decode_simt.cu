@@ -30,9 +30,11 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
   int g = g0;
   while (g < g1) {
     const int it = plan.item_of_tile(g);
-    const int a = prm.prefix[it], e = prm.prefix[it + 1];
-    const int t0 = g - a, t1 = min(e, g1) - a;
-    g = a + t1;
+    const int a = plan.first_tile(it), e = prm.prefix[it + 1];
+    const int lo = max(g, a), hi = min(e, g1);
+    g = min(e, g1);
+    if (hi <= lo) continue;                  // only overhead positions of this item fell into the part
+    const int t0 = lo - a, t1 = hi - a;
     const int b = it / prm.nrb, rb = it % prm.nrb;
     const int r0 = rb * kRowBlock;
     const int nrows = min(kRowBlock, prm.R - r0);

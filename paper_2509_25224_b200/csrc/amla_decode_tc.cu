@@ -97,12 +97,16 @@ struct UnitIter {
     else { g = plan.part_start(p); g1 = plan.part_start(p + 1); }
   }
   __device__ bool next(Unit& u) {
-    if (g >= g1) return false;
-    const int it = plan.item_of_tile(g);
-    const int a = prm.prefix[it], e = prm.prefix[it + 1];
-    u.t0 = g - a;
-    u.t1 = min(e, g1) - a;
-    g = a + u.t1;
+    int it, a;
+    while (true) {
+      if (g >= g1) return false;
+      it = plan.item_of_tile(g);
+      a = plan.first_tile(it);
+      const int e = prm.prefix[it + 1];
+      const int lo = max(g, a), hi = min(e, g1);
+      g = min(e, g1);
+      if (hi > lo) { u.t0 = lo - a; u.t1 = hi - a; break; }   // else: only overhead positions of this item fell into the part
+    }
     u.b = it / prm.nrb;
     u.r0 = (it % prm.nrb) * kRowBlock;
     u.nrows = min(kRowBlock, prm.R - u.r0);

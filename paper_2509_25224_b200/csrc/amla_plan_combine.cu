@@ -6,7 +6,8 @@
 
 namespace amla {
 
-// One block.  prefix[it] = sum over items before `it` of ceil(seqlens[b(it)] / 64); also resets the
+// One block.  prefix[it] = sum over items before `it` of their schedule lengths (tiles plus the start-up
+// overhead of a non-empty item, see Plan); also resets the
 // status word.  n_items is small (B * ceil(Sq*H/128)); a chunked block scan covers any size.
 __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_items,
                             int* __restrict__ prefix, int* __restrict__ status) {
@@ -23,6 +24,7 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
       int n = seqlens[it / nrb];
       n = n < 0 ? 0 : n;
       v = (n + kPage - 1) / kPage;
+      if (v > 0) v += kUnitOverheadTiles;
     }
     int x = v;  // inclusive warp scan
     for (int o = 1; o < 32; o <<= 1) {

@@ -10,6 +10,7 @@ import pytest
 from paper_2509_25224_b200 import binding, build, synth
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+UNIT_OVERHEAD = 10      # kUnitOverheadTiles of the schedule
 
 
 @pytest.fixture(scope="module")
@@ -86,9 +87,15 @@ def _check_plan(seqlens, Sq, H, P):
             assert all(s >= 0 for _, s, _ in parts)
             ps = [p for p, _, _ in parts]
             assert ps == list(range(ps[0], ps[0] + len(ps)))   # consecutive parts
-    L = sum(tiles)
-    if L:
-        assert per_part.max() - per_part.min() <= 1     # balanced to one tile
+    # balance: the schedule cuts a range in which every non-empty item is preceded by UNIT_OVERHEAD positions
+    # (the cost of starting an item) into equal parts, so no part holds more tiles than one such share
+    Lv = sum(t + UNIT_OVERHEAD for t in tiles if t)
+    if Lv:
+        assert per_part.max() <= -(-Lv // min(P, Lv))
+        starts = np.zeros(P, dtype=np.int64)            # items whose first tile a part holds
+        for p, it, t0, t1, slot, ns in units:
+            starts[p] += t0 == 0
+        assert (per_part + UNIT_OVERHEAD * starts).max() <= -(-Lv // min(P, Lv)) + UNIT_OVERHEAD
     return units
 
 
@@ -107,7 +114,8 @@ def test_plan_covers_every_tile_once_and_balances(lib, P):
 
 
 def test_plan_small_case_by_hand(lib):
-    # two sequences of 3 and 1 tiles, 2 parts: linear tiles [0,1,2 | 3]; part 0 = [0,2), part 1 = [2,4)
+    # two sequences of 3 and 1 tiles, 2 parts: positions [10 overhead, tiles 0-2 | 10 overhead, tile 0] = 24;
+    # part 0 = [0,12) holds tiles 0,1 of the first item, part 1 = [12,24) its tile 2 and the second item
     u = binding.plan_host(np.array([129, 10]), 1, 128, 2)
     assert u.tolist() == [[0, 0, 0, 2, 0, 2], [1, 0, 2, 3, 2, 2], [1, 1, 0, 1, -1, 1]]
 
