@@ -168,10 +168,14 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   const bool simt = (flags & AMLA_FLAG_KERNEL_SIMT) != 0;
   prm.P = simt ? sms : decode_tc_parts(sms);
 
+  prm.fused_plan = (!simt && n_items <= kFusedPlanMaxItems) ? 1 : 0;
+
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   profile_mark(0, stream);
-  if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-  ++g_last_launches;
+  if (!prm.fused_plan) {
+    if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+    ++g_last_launches;
+  }
   profile_mark(1, stream);
   if (simt) {
     if (launch_decode_simt(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }

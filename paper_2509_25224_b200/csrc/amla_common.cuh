@@ -38,6 +38,7 @@ struct DecodeParams {
   int n_items;                   // B * nrb
   int num_blocks, max_blocks_per_seq;
   int P;                         // parts the linear tile range is cut into
+  int fused_plan;                // the decode kernel computes `prefix` itself (few items), no schedule kernel
   int flags;
   unsigned long long* trace;     // timeline buffer of a -DAMLA_TRACE build, else unused (nullptr)
 };
@@ -67,6 +68,14 @@ constexpr int kTraceTiles = 96;
 // tiles whose positions it owns; overhead positions carry no work.
 // ---------------------------------------------------------------------------------------------
 constexpr int kUnitOverheadTiles = 10;
+constexpr int kFusedPlanMaxItems = 2048;   // up to this many items every decode CTA computes the prefix itself
+
+// Schedule length of an item: its tiles plus the start-up overhead (nothing for an empty sequence).
+__host__ __device__ inline int schedule_length(int seqlen) {
+  const int n = seqlen < 0 ? 0 : seqlen;
+  const int tiles = (n + kPage - 1) / kPage;
+  return tiles > 0 ? tiles + kUnitOverheadTiles : 0;
+}
 
 struct Plan {
   const int* prefix;

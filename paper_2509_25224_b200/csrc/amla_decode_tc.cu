@@ -227,10 +227,37 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   const uint32_t tbase = ld_shared_b32(tmem_slot);
   if (tid == 0) AMLA_STAMP(prm, part, is_score ? 0 : 1, 0);
 
-  // Launched with programmatic stream serialization: everything above ran while the schedule kernel was still
-  // going; its prefix array (and the caller's earlier work on the stream) is visible after this wait.
+  // Launched with programmatic stream serialization: everything above ran while the kernel before this one on the
+  // stream was still going; its results (the schedule kernel's prefix array, or the previous call's reads of the
+  // workspace) are complete after this wait.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
+  if (prm.fused_plan) {
+    // Few items: every CTA computes the schedule prefix itself (all write the same values; the combine kernel
+    // reads them later) instead of waiting for a one-block kernel.  Warp 6 scans 32 items at a time.
+    if (wid == 6) {
+      int* pw = const_cast<int*>(prm.prefix);
+      int carry = 0;
+      for (int base = 0; base < prm.n_items; base += 32) {
+        const int it = base + lane;
+        const int v = it < prm.n_items ? schedule_length(prm.seqlens[it / prm.nrb]) : 0;
+        int x = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, x, o);
+          if (lane >= o) x += y;
+        }
+        if (it < prm.n_items) pw[it] = carry + x - v;
+        carry += __shfl_sync(0xffffffffu, x, 31);
+      }
+      if (lane == 0) {
+        pw[prm.n_items] = carry;
+        if (blockIdx.x == 0) *prm.status = kStatusOk;
+      }
+      __threadfence_block();
+    }
+    __syncthreads();
+  }
   if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
     UnitIter first(prm, part);
     Unit fu;

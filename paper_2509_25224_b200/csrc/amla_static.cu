@@ -124,10 +124,12 @@ extern "C" int amla_mla_decode_static(const void* q, const void* kv_cache, const
   prm.tau = static_cast<float>(AMLA_DEFAULT_TAU);
   prm.P = parts;
 
-  // Nothing in the scratch has to be cleared by the host: the first kernel rewrites the status word and the whole
+  // Nothing in the scratch has to be cleared by the host: the first kernel (the schedule kernel, or for few items the
+  // decode kernel itself) rewrites the status word and the whole
   // prefix, and every partial that the combine reads is written by the decode kernel of the same call.
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  prm.fused_plan = prm.n_items <= kFusedPlanMaxItems ? 1 : 0;
+  if (!prm.fused_plan && launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
   int unsupported = 0;
   if (launch_decode_tc(prm, stream, &unsupported) != cudaSuccess) {
     cudaGetLastError();

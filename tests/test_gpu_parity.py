@@ -52,6 +52,13 @@ def test_many_short_sequences_more_items_than_parts():
     check_full(w)
 
 
+def test_more_items_than_the_in_kernel_schedule_handles():
+    # above 2048 (sequence, row block) items the schedule prefix comes from its own kernel instead of the decode kernel
+    rng = np.random.default_rng(10)
+    w = synth.make_workload("big", 2100, 1, 16, rng.integers(0, 130, 2100), seed=11)
+    check_full(w)
+
+
 @pytest.mark.parametrize("mode", MODES)
 def test_staircase_rescale(mode):
     check_full(synth.config_stress(B=2, N=4096), mode)
