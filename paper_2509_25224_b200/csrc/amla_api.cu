@@ -249,10 +249,7 @@ extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int 
   int acc = 0;
   for (int it = 0; it < n_items; ++it) {
     prefix[it] = acc;
-    int n = seqlens[it / nrb];
-    if (n < 0) n = 0;
-    const int tiles = (n + kPage - 1) / kPage;
-    acc += tiles > 0 ? tiles + kUnitOverheadTiles : 0;
+    acc += schedule_length(seqlens[it / nrb], it);
   }
   prefix[n_items] = acc;
   const Plan plan = Plan::make(prefix, n_items, num_parts);

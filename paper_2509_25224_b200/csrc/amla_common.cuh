@@ -62,19 +62,22 @@ constexpr int kTraceTiles = 96;
 // Split-KV schedule.  Items (sequence b, row block rb) in order it = b * nrb + rb own
 // ceil(N_b / 64) tiles each.  Starting an item costs a cluster a fixed amount of time (its Q rows,
 // the pipeline fill, the epilogue) that is worth about kUnitOverheadTiles tiles, so the schedule
-// balances a linear range in which every non-empty item is preceded by that many overhead
-// positions: prefix[it] is the position where item `it` begins (overhead first, then its tiles),
+// balances a linear range in which every non-empty item but the first is preceded by that many
+// overhead positions: prefix[it] is the position where item `it` begins (overhead first, then its tiles),
 // L = prefix[n_items] the total, and part p owns positions [p*L/P, (p+1)*L/P).  A part does the
 // tiles whose positions it owns; overhead positions carry no work.
 // ---------------------------------------------------------------------------------------------
 constexpr int kUnitOverheadTiles = 10;
 constexpr int kFusedPlanMaxItems = 2048;   // up to this many items every decode CTA computes the prefix itself
 
+// Overhead positions in front of item `it`: none for the first item, which opens the first part anyway (every
+// part pays for one start; the positions stand for the additional ones).
+__host__ __device__ inline int item_overhead(int it) { return it > 0 ? kUnitOverheadTiles : 0; }
 // Schedule length of an item: its tiles plus the start-up overhead (nothing for an empty sequence).
-__host__ __device__ inline int schedule_length(int seqlen) {
+__host__ __device__ inline int schedule_length(int seqlen, int it) {
   const int n = seqlen < 0 ? 0 : seqlen;
   const int tiles = (n + kPage - 1) / kPage;
-  return tiles > 0 ? tiles + kUnitOverheadTiles : 0;
+  return tiles > 0 ? tiles + item_overhead(it) : 0;
 }
 
 struct Plan {
@@ -113,7 +116,7 @@ struct Plan {
     return lo;
   }
   // Position of the first tile of a non-empty item.
-  __host__ __device__ int first_tile(int it) const { return prefix[it] + kUnitOverheadTiles; }
+  __host__ __device__ int first_tile(int it) const { return prefix[it] + item_overhead(it); }
   // Parts [p_first, p_last] that hold tiles of item `it`; returns the split count (0 for an empty item).
   __host__ __device__ int item_parts(int it, int* p_first, int* p_last) const {
     const int e = prefix[it + 1];

@@ -240,7 +240,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       int carry = 0;
       for (int base = 0; base < prm.n_items; base += 32) {
         const int it = base + lane;
-        const int v = it < prm.n_items ? schedule_length(prm.seqlens[it / prm.nrb]) : 0;
+        const int v = it < prm.n_items ? schedule_length(prm.seqlens[it / prm.nrb], it) : 0;
         int x = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {

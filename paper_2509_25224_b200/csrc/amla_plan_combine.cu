@@ -20,7 +20,7 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
   for (int base = 0; base < n_items; base += blockDim.x) {
     const int it = base + tid;
     int v = 0;
-    if (it < n_items) v = schedule_length(seqlens[it / nrb]);
+    if (it < n_items) v = schedule_length(seqlens[it / nrb], it);
     int x = v;  // inclusive warp scan
     for (int o = 1; o < 32; o <<= 1) {
       int y = __shfl_up_sync(0xffffffffu, x, o);

@@ -87,9 +87,9 @@ def _check_plan(seqlens, Sq, H, P):
             assert all(s >= 0 for _, s, _ in parts)
             ps = [p for p, _, _ in parts]
             assert ps == list(range(ps[0], ps[0] + len(ps)))   # consecutive parts
-    # balance: the schedule cuts a range in which every non-empty item is preceded by UNIT_OVERHEAD positions
+    # balance: the schedule cuts a range in which every non-empty item but the first is preceded by UNIT_OVERHEAD positions
     # (the cost of starting an item) into equal parts, so no part holds more tiles than one such share
-    Lv = sum(t + UNIT_OVERHEAD for t in tiles if t)
+    Lv = sum(t + (UNIT_OVERHEAD if it else 0) for it, t in enumerate(tiles) if t)
     if Lv:
         assert per_part.max() <= -(-Lv // min(P, Lv))
         starts = np.zeros(P, dtype=np.int64)            # items whose first tile a part holds
@@ -114,10 +114,10 @@ def test_plan_covers_every_tile_once_and_balances(lib, P):
 
 
 def test_plan_small_case_by_hand(lib):
-    # two sequences of 3 and 1 tiles, 2 parts: positions [10 overhead, tiles 0-2 | 10 overhead, tile 0] = 24;
-    # part 0 = [0,12) holds tiles 0,1 of the first item, part 1 = [12,24) its tile 2 and the second item
+    # two sequences of 3 and 1 tiles, 2 parts: positions [tiles 0-2 | 10 overhead, tile 0] = 14; part 0 = [0,7) holds
+    # the first item, part 1 = [7,14) the second
     u = binding.plan_host(np.array([129, 10]), 1, 128, 2)
-    assert u.tolist() == [[0, 0, 0, 2, 0, 2], [1, 0, 2, 3, 2, 2], [1, 1, 0, 1, -1, 1]]
+    assert u.tolist() == [[0, 0, 0, 3, -1, 1], [1, 1, 0, 1, -1, 1]]
 
 
 def test_batch_sharding_partitions_sequences():
