@@ -28,11 +28,12 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_trace() -> str:
-    """Developer aid: libamla_trace.so, the same sources with -DAMLA_TRACE (per-role cycle stamps)."""
+def build_trace(level: int = 1) -> str:
+    """Developer aid: libamla_trace.so, the same sources with -DAMLA_TRACE=level (per-role cycle stamps;
+    level 2 adds several stamps per ring slot, which slows the issuer loops it measures)."""
     out = os.path.join(_HERE, "libamla_trace.so")
     nvcc = os.environ.get("NVCC", "nvcc")
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")] + ["-DAMLA_TRACE"]
+    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")] + [f"-DAMLA_TRACE={level}"]
     subprocess.check_call([nvcc] + flags + sources() + ["-o", out])
     return out
 
@@ -53,6 +54,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 if __name__ == "__main__":
     if "--trace" in sys.argv:
-        print(build_trace())
+        print(build_trace(2 if "--full" in sys.argv else 1))
         sys.exit(0)
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

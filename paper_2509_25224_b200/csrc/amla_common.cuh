@@ -57,6 +57,12 @@ constexpr int kTraceTiles = 96;
 #else
 #define AMLA_STAMP(prm, part, ev, idx) do { } while (0)
 #endif
+// Detailed stamps (several per ring slot) perturb the issuer loops; -DAMLA_TRACE=2 turns them on.
+#if defined(AMLA_TRACE) && AMLA_TRACE >= 2
+#define AMLA_STAMP2(prm, part, ev, idx) AMLA_STAMP(prm, part, ev, idx)
+#else
+#define AMLA_STAMP2(prm, part, ev, idx) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // Split-KV schedule.  Items (sequence b, row block rb) in order it = b * nrb + rb own

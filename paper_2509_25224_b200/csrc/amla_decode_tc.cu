@@ -311,7 +311,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
-          if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
+          if (tid == 0) AMLA_STAMP2(prm, part, 5, gt);
           const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
           const bool masked = t + npages > first_masked_tile;
           const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
@@ -362,7 +362,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
               if (h == npages - 1) {       // the score tile has been read for the last time
                 tc_fence_before_sync();
                 mbar_arrive(bar(A_SEMPTY + sb));
-                if (tid == 0) AMLA_STAMP(prm, part, 6, gt);
+                if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
               }
               uint32_t pk[32];
               if (masked) {
@@ -387,11 +387,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
               }
               // stage P~ and N; the copy warps ship them to the value CTA
               const uint32_t s2 = gt & 1;
-              if (tid == 0) AMLA_STAMP(prm, part, 7, gt);
+              if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
               // one staging buffer: the copy warps of the previous page must have read it into registers
               if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
               if (!ok) break;
-              if (tid == 0) AMLA_STAMP(prm, part, 8, gt);
+              if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
               const uint32_t stg = smem_base + kOffStage;
 #pragma unroll
               for (int c = 0; c < 8; ++c)
@@ -452,7 +452,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             }
           }
           if (have && mbar_probe(my_empty, par)) {
-            AMLA_STAMP(prm, part, 20, issued * kNumKSlots + lane);
+            AMLA_STAMP2(prm, part, 20, issued * kNumKSlots + lane);
             mbar_arrive_expect_tx(my_full, npages * kKPageBytes);
             tma_load_4d(dst, &kv_map, 0, 0, 3 * g, page0 * 8, my_full);
             if (npages > 1) tma_load_4d(dst + kKPageBytes, &kv_map, 0, 0, 3 * g, page1 * 8, my_full);
@@ -495,33 +495,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             ok = mbar_wait(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
-            AMLA_STAMP(prm, part, 3, gt);
+            AMLA_STAMP2(prm, part, 3, gt);
             const uint32_t d = tbase + kSCol + 128 * sb;
-            uint32_t qa = tbase + kQCol;          // A operand: eight tensor-memory columns per K = 16 step
-            uint32_t acc = 0;
-#pragma unroll 1
+            // Written out per slot and column block, so that every accumulate flag, operand offset and trip count
+            // is a compile-time constant: with run-time trip counts the same loop issued 25 % slower.
+#pragma unroll
             for (int g = 0; g < 3; ++g) {
-              AMLA_STAMP(prm, part, 25, gc);
-              ok = mbar_wait(bar(A_KFULL) + 8 * slot, kpar);    // TMA data -> MMA operand: both async proxy, no fence needed
-              if (!ok) break;
-              AMLA_STAMP(prm, part, 21, gc);
-              uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
-              const int n_blk = g < 2 ? 3 : 2;     // the last column block takes the RoPE columns of Q from shared memory
-#pragma unroll 1
-              for (int cl = 0; cl < n_blk; ++cl) {
+              AMLA_STAMP2(prm, part, 25, gc);
+              ok = ok && mbar_wait(bar(A_KFULL) + 8 * slot, kpar);    // TMA data -> MMA operand: both async proxy, no fence needed
+              if (ok) {
+                AMLA_STAMP2(prm, part, 21, gc);
+                const uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ts(d, qa + 8 * kk, smem_desc_join(klo + 2 * kk, dhi), idesc, kk == 0 ? acc : 1u);
-                acc = 1;
-                qa += 32;
-                klo += 64;
-              }
-              if (g == 2) {
+                for (int cl = 0; cl < 3; ++cl) {
+                  const int c = 3 * g + cl;
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ss(d, smem_desc_join(qlo0 + 2 * kk, qhi), smem_desc_join(klo + 2 * kk, dhi), idesc, 1u);
+                  for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t bd = smem_desc_join(klo + 64 * cl + 2 * kk, dhi);
+                    if (c < 8) mma_ts(d, tbase + kQCol + 32 * c + 8 * kk, bd, idesc, (c | kk) != 0 ? 1u : 0u);
+                    else mma_ss(d, smem_desc_join(qlo0 + 2 * kk, qhi), bd, idesc, 1u);   // RoPE columns: Q from shared memory
+                  }
+                }
+                AMLA_STAMP2(prm, part, 26, gc);
+                mma_commit(bar(A_KEMPTY) + 8 * slot);
+                AMLA_STAMP2(prm, part, 22, gc);
               }
-              AMLA_STAMP(prm, part, 26, gc);
-              mma_commit(bar(A_KEMPTY) + 8 * slot);
-              AMLA_STAMP(prm, part, 22, gc);
               ++gc;
               if (++slot == kNumKSlots) { slot = 0; kpar ^= 1; }
             }
@@ -549,7 +547,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         const uint64_t t_start = global_timer_ns();
         for (uint32_t spin = 0;; ++spin) {
           const bool act = lane < kNumKSlots && g < total;
-          if (act && mbar_probe(bar(A_KFULL + lane), par)) { AMLA_STAMP(prm, part, 24, g); g += kNumKSlots; par ^= 1; }
+          if (act && mbar_probe(bar(A_KFULL + lane), par)) { AMLA_STAMP2(prm, part, 24, g); g += kNumKSlots; par ^= 1; }
           if (!__any_sync(0xffffffffu, act)) break;
           if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) break;
         }
@@ -607,7 +605,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             if (!ok) break;
             const uint32_t pfull = peerB_bars + 8u * (B_PFULL + pb);
             const uint32_t dst = peerB_base + kOffP + pb * kPStride + (half * kChunks * 32 + lane) * 16;
-            if (lane == 0 && half == 0) { AMLA_STAMP(prm, part, 23, gt); mbar_arrive_expect_tx_cluster(pfull, kPXfer); }
+            if (lane == 0 && half == 0) { AMLA_STAMP2(prm, part, 23, gt); mbar_arrive_expect_tx_cluster(pfull, kPXfer); }
 #pragma unroll
             for (int i = 0; i < kChunks; ++i) {
               if (half * kChunks + i < 33) st_async_v4(dst + i * 512, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
@@ -629,7 +627,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           const uint32_t s = gt % kNumP, k = gt / kNumP;
           ok = warp_wait<true>(bar(B_PFULL + s), k & 1);
           if (!ok) break;
-          if (tid == 0) AMLA_STAMP(prm, part, 13, gt);
+          if (tid == 0) AMLA_STAMP2(prm, part, 13, gt);
           const uint32_t nword = ld_shared_b32(smem_base + kOffP + s * kPStride + kPBytes + r * 4);
           const bool mine = (kMode == 2) ? (__uint_as_float(nword) != 1.f) : (nword != 0u);
           if (__any_sync(0xffffffffu, mine) && t > u.t0) {
@@ -666,7 +664,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             tc_fence_before_sync();
           }
           mbar_arrive(bar(B_OREADY + s));
-          if (tid == 0) AMLA_STAMP(prm, part, 14, gt);
+          if (tid == 0) AMLA_STAMP2(prm, part, 14, gt);
         }
         if (!ok) break;
         // ---- epilogue (line 20): out = O / (l * S16)
@@ -771,7 +769,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             }
           }
           if (have && mbar_probe(my_empty, par)) {
-            if ((my_gv & 1) == 0) AMLA_STAMP(prm, part, 12, my_gv >> 1);
+            if ((my_gv & 1) == 0) AMLA_STAMP2(prm, part, 12, my_gv >> 1);
             mbar_arrive_expect_tx(my_full, kVSlotBytes);
             tma_load_3d(dst, &v_map, 0, page * kPage, (my_gv & 1) * 4, my_full);
             my_gv += kNumVSlots;
@@ -810,7 +808,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             for (int nh = 0; nh < 2; ++nh) {
               ok = mbar_wait(bar(B_VFULL) + 8 * slot, vpar);
               if (!ok) break;
-              if (nh == 0) AMLA_STAMP(prm, part, 15, gt);
+              if (nh == 0) AMLA_STAMP2(prm, part, 15, gt);
               uint32_t vlo = vlo0 + slot * (kVSlotBytes >> 4);
               uint32_t pl = plo;
               uint32_t acc = acc0;
