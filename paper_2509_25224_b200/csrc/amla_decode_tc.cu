@@ -377,13 +377,22 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                   pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
                 }
               } else {
+                // two elements per instruction (packed FP32 pairs) for the scale-and-subtract, the row sum and the S16 scaling
+                const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
+                const uint64_t ps2 = pack_f32x2(sp.p_scale, sp.p_scale);
+                uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                  const float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
-                  const float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
-                  rs0 += p0; rs1 += p1;
-                  pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+                  float x0, x1, q0, q1;
+                  unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1])), sc2, ns2), x0, x1);
+                  const uint64_t pp = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
+                  if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
+                  unpack_f32x2(mul_f32x2(pp, ps2), q0, q1);
+                  pk[i] = pack_bf16x2(q0, q1);
                 }
+                float s0, s1;
+                unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
+                rs0 += s0; rs1 += s1;
               }
               // stage P~ and N; the copy warps ship them to the value CTA
               const uint32_t s2 = gt & 1;
