@@ -311,7 +311,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
           if (!ok) break;
           tc_fence_after_sync();
-          if (tid == 0) AMLA_STAMP2(prm, part, 5, gt);
+          if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
           const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
           const bool masked = t + npages > first_masked_tile;
           const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
@@ -504,7 +504,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             ok = mbar_wait(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
-            AMLA_STAMP2(prm, part, 3, gt);
+            AMLA_STAMP(prm, part, 3, gt);
             const uint32_t d = tbase + kSCol + 128 * sb;
             // Written out per slot and column block, so that every accumulate flag, operand offset and trip count
             // is a compile-time constant: with run-time trip counts the same loop issued 25 % slower.
