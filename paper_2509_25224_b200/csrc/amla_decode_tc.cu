@@ -316,104 +316,103 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           const bool masked = t + npages > first_masked_tile;
           const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
 
+          // The S tile is read from tensor memory in 32-column chunks, twice (maximum, then exponentials); the load
+          // of the next chunk is always in flight while a chunk is processed, so that the TMEM latency is hidden.
+          uint32_t b0[32], b1[32];
           // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
           float ext = scale_nonneg ? -INFINITY : INFINITY;
-#pragma unroll 1
-          for (int h = 0; h < 2; ++h) {
-            if (h < npages) {
-              uint32_t lo[32], hi[32];
-              tmem_ld_32x32b_x32(scol + 64 * h, lo);
-              tmem_ld_32x32b_x32(scol + 64 * h + 32, hi);
-              tmem_wait_ld();
-              if (masked) {
+          auto chunk_max = [&](uint32_t (&v)[32], int col0) {
+            if (masked) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                  lo[i] = (64 * h + i < nvis) ? lo[i] : mask_fill;
-                  hi[i] = (64 * h + 32 + i < nvis) ? hi[i] : mask_fill;
-                }
-              }
-              if (scale_nonneg) {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) ext = fmax3(ext, __uint_as_float(lo[i]), __uint_as_float(hi[i]));
-              } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) ext = fminf(ext, fminf(__uint_as_float(lo[i]), __uint_as_float(hi[i])));
-              }
+              for (int i = 0; i < 32; ++i) v[i] = (col0 + i < nvis) ? v[i] : mask_fill;
             }
+            if (scale_nonneg) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) ext = fmax3(ext, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) ext = fminf(ext, fminf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+            }
+          };
+          tmem_ld_32x32b_x32(scol, b0);
+#pragma unroll 1
+          for (int h = 0; h < npages; ++h) {
+            tmem_wait_ld();
+            tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+            chunk_max(b0, 64 * h);
+            tmem_wait_ld();
+            tmem_ld_32x32b_x32(scol + (h + 1 < npages ? 64 * (h + 1) : 0), b0);   // next half, or the first chunk again for the second pass
+            chunk_max(b1, 64 * h + 32);
           }
           const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
           const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
           const float nsub = -sp.m2_sub;
           float rs0 = 0.f, rs1 = 0.f;
-
-          // lines 6, 10 per 64-key half: P, row sum (FP32, unscaled), P~ = bf16(P * S16)
-#pragma unroll 1
-          for (int h = 0; h < 2; ++h) {
-            if (h < npages) {
-              uint32_t a[64];
-              {
-                uint32_t lo[32], hi[32];
-                tmem_ld_32x32b_x32(scol + 64 * h, lo);
-                tmem_ld_32x32b_x32(scol + 64 * h + 32, hi);
-                tmem_wait_ld();
+          const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
+          const uint64_t ps2 = pack_f32x2(sp.p_scale, sp.p_scale);
+          uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
+          uint32_t pk[32];
+          // lines 6, 10 for 32 columns: P, row sum (FP32, unscaled), P~ = bf16(P * S16), two elements per instruction
+          auto chunk_exp = [&](const uint32_t (&v)[32], int col0, int k0) {
+            if (masked) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) { a[i] = lo[i]; a[32 + i] = hi[i]; }
+              for (int i = 0; i < 16; ++i) {
+                float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, nsub));
+                float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, nsub));
+                p0 = (col0 + 2 * i < nvis) ? p0 : 0.f;
+                p1 = (col0 + 2 * i + 1 < nvis) ? p1 : 0.f;
+                rs0 += p0; rs1 += p1;
+                pk[k0 + i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
               }
-              if (h == npages - 1) {       // the score tile has been read for the last time
-                tc_fence_before_sync();
-                mbar_arrive(bar(A_SEMPTY + sb));
-                if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                float x0, x1, q0, q1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, ns2), x0, x1);
+                const uint64_t pp = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
+                if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
+                unpack_f32x2(mul_f32x2(pp, ps2), q0, q1);
+                pk[k0 + i] = pack_bf16x2(q0, q1);
               }
-              uint32_t pk[32];
-              if (masked) {
-                const int nv = nvis - 64 * h;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                  float p0 = ex2_approx(fmaf(__uint_as_float(a[2 * i]), prm.scale_log2, nsub));
-                  float p1 = ex2_approx(fmaf(__uint_as_float(a[2 * i + 1]), prm.scale_log2, nsub));
-                  p0 = (2 * i < nv) ? p0 : 0.f;
-                  p1 = (2 * i + 1 < nv) ? p1 : 0.f;
-                  rs0 += p0; rs1 += p1;
-                  pk[i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
-                }
-              } else {
-                // two elements per instruction (packed FP32 pairs) for the scale-and-subtract, the row sum and the S16 scaling
-                const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
-                const uint64_t ps2 = pack_f32x2(sp.p_scale, sp.p_scale);
-                uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                  float x0, x1, q0, q1;
-                  unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1])), sc2, ns2), x0, x1);
-                  const uint64_t pp = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
-                  if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
-                  unpack_f32x2(mul_f32x2(pp, ps2), q0, q1);
-                  pk[i] = pack_bf16x2(q0, q1);
-                }
-                float s0, s1;
-                unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
-                rs0 += s0; rs1 += s1;
-              }
-              // stage P~ and N; the copy warps ship them to the value CTA
-              const uint32_t s2 = gt & 1;
-              if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
-              // one staging buffer: the copy warps of the previous page must have read it into registers
-              if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
-              if (!ok) break;
-              if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
-              const uint32_t stg = smem_base + kOffStage;
-#pragma unroll
-              for (int c = 0; c < 8; ++c)
-                st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-              // the rescale (if any) belongs to the first half; the second half leaves O alone
-              const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
-                                                  : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
-              st_shared_b32(stg + kPBytes + r * 4, nword);
-              fence_proxy_async_smem();
-              mbar_arrive(bar(A_PSTAGED + s2));
-              if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
-              ++gt;
             }
+          };
+#pragma unroll 1
+          for (int h = 0; h < npages; ++h) {
+            tmem_wait_ld();
+            tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+            chunk_exp(b0, 64 * h, 0);
+            tmem_wait_ld();
+            if (h + 1 < npages) {
+              tmem_ld_32x32b_x32(scol + 64 * (h + 1), b0);
+            } else {                       // the score tile has been read for the last time
+              tc_fence_before_sync();
+              mbar_arrive(bar(A_SEMPTY + sb));
+              if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
+            }
+            chunk_exp(b1, 64 * h + 32, 16);
+            // stage P~ and N; the copy warps ship them to the value CTA
+            const uint32_t s2 = gt & 1;
+            if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
+            // one staging buffer: the copy warps of the previous page must have read it into registers
+            if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+            if (!ok) break;
+            if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
+            const uint32_t stg = smem_base + kOffStage;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            // the rescale (if any) belongs to the first half; the second half leaves O alone
+            const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
+                                                : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
+            st_shared_b32(stg + kPBytes + r * 4, nword);
+            mbar_arrive(bar(A_PSTAGED + s2));
+            if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
+            ++gt;
+          }
+          {
+            float s0, s1;
+            unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
+            rs0 += s0; rs1 += s1;
           }
           st.l = st.l * sp.l_up + (rs0 + rs1);
         }
@@ -446,6 +445,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane);
         const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
         const uint64_t t_start = global_timer_ns();
+        bool progress = false;
         for (uint32_t spin = 0;; ++spin) {
           if (!fin && !have) {
             int lt;
@@ -471,8 +471,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             par ^= 1;
             ++issued;
             have = false;
+            progress = true;
           }
           if (__all_sync(0xffffffffu, fin)) break;
+          // nothing to issue right now: back off, so that the polling does not take issue slots from the warps that
+          // share this scheduler
+          if (!__any_sync(0xffffffffu, progress)) __nanosleep(100);
+          progress = false;
           if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > 4 * kWaitLimitNs)) { ok = false; break; }
         }
         if (!ok) {
@@ -767,6 +772,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         const uint32_t my_full = bar(B_VFULL + lane), my_empty = bar(B_VEMPTY + lane);
         const uint32_t dst = smem_base + kOffV + lane * kVSlotBytes;
         const uint64_t t_start = global_timer_ns();
+        bool progress = false;
         for (uint32_t spin = 0;; ++spin) {
           if (!fin && !have) {
             int lt;
@@ -785,8 +791,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             par ^= 1;
             ++issued;
             have = false;
+            progress = true;
           }
           if (__all_sync(0xffffffffu, fin)) break;
+          // nothing to issue right now: back off, so that the polling does not take issue slots from the warps that
+          // share this scheduler
+          if (!__any_sync(0xffffffffu, progress)) __nanosleep(100);
+          progress = false;
           if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > 4 * kWaitLimitNs)) { ok = false; break; }
         }
         if (!ok) {
