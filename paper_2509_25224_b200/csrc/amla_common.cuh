@@ -91,6 +91,7 @@ struct Plan {
   int n_items;
   int L;
   int P;
+  bool wide;     // L * P does not fit 31 bits: the part arithmetic needs 64-bit division (slow on the device)
 
   // With fewer positions than parts only the first L parts exist (one position each).
   __host__ __device__ static Plan make(const int* prefix, int n_items, int max_parts) {
@@ -99,14 +100,20 @@ struct Plan {
     pl.n_items = n_items;
     pl.L = prefix[n_items];
     pl.P = pl.L < max_parts ? (pl.L > 0 ? pl.L : 1) : max_parts;
+    pl.wide = static_cast<long long>(pl.L) * pl.P >= (1ll << 31);
     return pl;
+  }
+  // floor(a * b / c) for 0 <= a <= c-ish operands of the schedule; 32-bit unless the product could overflow
+  __host__ __device__ int muldiv(int a, int b, int c) const {
+    if (!wide) return static_cast<int>(static_cast<unsigned>(a) * static_cast<unsigned>(b) / static_cast<unsigned>(c));
+    return static_cast<int>((static_cast<long long>(a) * b) / c);
   }
   __host__ __device__ int part_start(int p) const {
     if (p >= P) return L;
-    return static_cast<int>((static_cast<long long>(p) * L) / P);
+    return muldiv(p, L, P);
   }
   __host__ __device__ int part_of_tile(int g) const {
-    int p = static_cast<int>((static_cast<long long>(g) * P) / L);
+    int p = muldiv(g, P, L);
     if (p > P - 1) p = P - 1;
     while (p + 1 < P && part_start(p + 1) <= g) ++p;
     while (p > 0 && part_start(p) > g) --p;
@@ -156,6 +163,12 @@ __device__ __forceinline__ float exponent_add_raw(float f, int n_bits) {
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float log2f_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 

@@ -64,7 +64,12 @@ constexpr uint32_t kEndB = kOffEpi + 4 * 32 * 128;
 // ---- both: the barriers sit at the same offset, so that one multicast commit can reach the two CTAs
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
 constexpr uint32_t kBarBytes = 512;
-constexpr uint32_t kSmemBytes = kOffBars + kBarBytes;
+// ---- both: a copy of the schedule prefix and of the sequence lengths for batches of up to kSmemPlanItems items,
+// so that the roles' schedule look-ups (a dozen dependent loads per unit) stay on chip
+constexpr int kSmemPlanItems = 128;
+constexpr uint32_t kOffPlan = kOffBars + kBarBytes;                          // int [kSmemPlanItems + 1] prefix
+constexpr uint32_t kOffSeqlens = kOffPlan + ((kSmemPlanItems + 1) * 4 + 15) / 16 * 16;   // int [kSmemPlanItems] sequence lengths
+constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
 static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
@@ -92,7 +97,9 @@ struct UnitIter {
   const DecodeParams& prm;
   Plan plan;
   int p, g, g1;
-  __device__ UnitIter(const DecodeParams& prm_, int part) : prm(prm_), plan(Plan::make(prm_.prefix, prm_.n_items, prm_.P)), p(part) {
+  const int* seqlens;
+  __device__ UnitIter(const DecodeParams& prm_, const int* prefix, const int* seqlens_, int part)
+      : prm(prm_), plan(Plan::make(prefix, prm_.n_items, prm_.P)), p(part), seqlens(seqlens_) {
     if (plan.L <= 0 || p >= plan.P) { g = g1 = 0; }
     else { g = plan.part_start(p); g1 = plan.part_start(p + 1); }
   }
@@ -102,7 +109,7 @@ struct UnitIter {
       if (g >= g1) return false;
       it = plan.item_of_tile(g);
       a = plan.first_tile(it);
-      const int e = prm.prefix[it + 1];
+      const int e = plan.prefix[it + 1];
       const int lo = max(g, a), hi = min(e, g1);
       g = min(e, g1);
       if (hi > lo) { u.t0 = lo - a; u.t1 = hi - a; break; }   // else: only overhead positions of this item fell into the part
@@ -110,7 +117,7 @@ struct UnitIter {
     u.b = it / prm.nrb;
     u.r0 = (it % prm.nrb) * kRowBlock;
     u.nrows = min(kRowBlock, prm.R - u.r0);
-    u.n_b = min(max(prm.seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
+    u.n_b = min(max(seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
     int p_first, p_last;
     const int nsplit = plan.item_parts(it, &p_first, &p_last);
     u.slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
@@ -126,7 +133,7 @@ struct Cursor {
   Unit u;
   int base;      // index of the current unit's first page / score tile
   bool valid;
-  __device__ Cursor(const DecodeParams& prm, int part) : it(prm, part), base(0) { valid = it.next(u); }
+  __device__ Cursor(const DecodeParams& prm, const int* prefix, const int* seqlens, int part) : it(prm, prefix, seqlens, part), base(0) { valid = it.next(u); }
   __device__ int count() const { return kTiles ? (u.t1 - u.t0 + 1) / 2 : (u.t1 - u.t0); }
   // false when k lies beyond the part's work; otherwise `local` is the index within the unit
   __device__ bool locate(int k, int& local) {
@@ -232,41 +239,52 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   // workspace) are complete after this wait.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
+  const int* prefix = prm.prefix;
+  const int* seqlens = prm.seqlens;
   if (prm.fused_plan) {
     // Few items: every CTA computes the schedule prefix itself (all write the same values; the combine kernel
-    // reads them later) instead of waiting for a one-block kernel.  Warp 6 scans 32 items at a time.
+    // reads them later) instead of waiting for a one-block kernel.  Warp 6 scans 32 items at a time.  A small
+    // batch's prefix and sequence lengths are also kept in shared memory, and the roles read those copies.
+    int* ps = prm.n_items <= kSmemPlanItems ? reinterpret_cast<int*>(smem_raw + kOffPlan) : nullptr;
     if (wid == 6) {
       int* pw = const_cast<int*>(prm.prefix);
       int carry = 0;
       for (int base = 0; base < prm.n_items; base += 32) {
         const int it = base + lane;
-        const int v = it < prm.n_items ? schedule_length(prm.seqlens[it / prm.nrb], it) : 0;
+        const int n_seq = it < prm.n_items ? prm.seqlens[it / prm.nrb] : 0;
+        if (ps && it < prm.n_items) reinterpret_cast<int*>(smem_raw + kOffSeqlens)[it / prm.nrb] = n_seq;   // same value from every row block
+        const int v = it < prm.n_items ? schedule_length(n_seq, it) : 0;
         int x = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           const int y = __shfl_up_sync(0xffffffffu, x, o);
           if (lane >= o) x += y;
         }
-        if (it < prm.n_items) pw[it] = carry + x - v;
+        if (it < prm.n_items) {
+          pw[it] = carry + x - v;
+          if (ps) ps[it] = carry + x - v;
+        }
         carry += __shfl_sync(0xffffffffu, x, 31);
       }
       if (lane == 0) {
         pw[prm.n_items] = carry;
+        if (ps) ps[prm.n_items] = carry;
         if (blockIdx.x == 0) *prm.status = kStatusOk;
       }
       __threadfence_block();
     }
     __syncthreads();
+    if (ps) { prefix = ps; seqlens = reinterpret_cast<const int*>(smem_raw + kOffSeqlens); }
   }
   if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
-    UnitIter first(prm, part);
+    UnitIter first(prm, prefix, seqlens, part);
     Unit fu;
     if (first.next(fu)) prefetch_q_row(prm, fu, tid);
   }
 
 
   bool ok = true;
-  UnitIter iter(prm, part);
+  UnitIter iter(prm, prefix, seqlens, part);
   Unit u;
   uint32_t gt = 0;      // 64-key pages processed by this cluster so far (all roles count identically)
   uint32_t un = 0;      // units processed so far
@@ -436,7 +454,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       // is still in use never holds up the loads of the others (one thread issuing a ring in order reaches a
       // fraction of the rate).
       {
-        Cursor<true> cur(prm, part);
+        Cursor<true> cur(prm, prefix, seqlens, part);
         int my_tile = lane / 3, g = lane % 3;   // score tile and column-block group of the next slot this lane loads
         uint32_t par = 1;                       // parity of the "empty" phase it has to see first
         bool fin = lane >= kNumKSlots, have = false;
@@ -552,7 +570,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     } else if (wid == 6 + kNumCopyWarps) {
       // trace builds: lane l watches K slot l and stamps the arrival of its data (non-blocking polls)
       if (prm.trace) {
-        Cursor<true> cur(prm, part);
+        Cursor<true> cur(prm, prefix, seqlens, part);
         int total = 0, lt;
         while (cur.valid) { total += cur.count(); cur.locate(total, lt); }
         total *= 3;
@@ -763,7 +781,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     } else if (wid == 4) {
       // ---- TMA producers: V, two slots (256 columns each, one 3-D box) per page; lane l owns ring slot l
       {
-        Cursor<false> cur(prm, part);
+        Cursor<false> cur(prm, prefix, seqlens, part);
         int my_gv = lane;                       // next slot of the sequence this lane loads (page = gv / 2)
         uint32_t par = 1;
         bool fin = lane >= kNumVSlots, have = false;
