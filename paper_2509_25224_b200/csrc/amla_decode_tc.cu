@@ -183,6 +183,161 @@ __device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int
   }
 }
 
+
+// What a role needs from the kernel's set-up.
+struct RoleCtx {
+  uint32_t smem_base, bars, tbase, peerB_bars, peerB_base;
+  const int* prefix;
+  const int* seqlens;
+  int part, tid;
+};
+
+// The softmax warpgroup's work on one unit: its score tiles, then the final scalars for the value CTA.  A function
+// of its own, so that it can also be run and timed outside the kernel.  Returns
+// (pages so far) << 32 | (score tiles so far) << 1 | ok.
+template <int kMode>
+__device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const RoleCtx c, const Unit u, uint32_t un, uint32_t gt, uint32_t gs) {
+  const int tid = c.tid, wid = tid >> 5, part = c.part;
+  const uint32_t smem_base = c.smem_base, bars = c.bars, tbase = c.tbase, peerB_bars = c.peerB_bars, peerB_base = c.peerB_base;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  (void)part;
+  bool ok = true;
+  const int r = tid;
+  const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+  const bool scale_nonneg = prm.scale_log2 >= 0.f;
+  const uint32_t mask_fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
+  {
+    RowState st;
+    row_state_init(st);
+    const int tok = (u.r0 + r) / prm.H;
+    const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);          // keys 0..visible-1 are seen by this row
+    const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // pages from here on may hold hidden keys
+
+    for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
+      const int npages = min(2, u.t1 - t);
+      const uint32_t sb = gs & 1;
+      ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
+      if (!ok) break;
+      tc_fence_after_sync();
+      if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
+      const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
+      const bool masked = t + npages > first_masked_tile;
+      const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
+
+      // The S tile is read from tensor memory in 32-column chunks, twice (maximum, then exponentials); the load
+      // of the next chunk is always in flight while a chunk is processed, so that the TMEM latency is hidden.
+      uint32_t b0[32], b1[32];
+      // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
+      float ext = scale_nonneg ? -INFINITY : INFINITY;
+      auto chunk_max = [&](uint32_t (&v)[32], int col0) {
+        if (masked) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = (col0 + i < nvis) ? v[i] : mask_fill;
+        }
+        if (scale_nonneg) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) ext = fmax3(ext, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) ext = fminf(ext, fminf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+        }
+      };
+      tmem_ld_32x32b_x32(scol, b0);
+#pragma unroll 1
+      for (int h = 0; h < npages; ++h) {
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+        chunk_max(b0, 64 * h);
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + (h + 1 < npages ? 64 * (h + 1) : 0), b0);   // next half, or the first chunk again for the second pass
+        chunk_max(b1, 64 * h + 32);
+      }
+      const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
+      const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
+      const float nsub = -sp.m2_sub;
+      float rs0 = 0.f, rs1 = 0.f;
+      const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
+      const uint64_t ps2 = pack_f32x2(sp.p_scale, sp.p_scale);
+      uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
+      uint32_t pk[32];
+      // lines 6, 10 for 32 columns: P, row sum (FP32, unscaled), P~ = bf16(P * S16), two elements per instruction
+      auto chunk_exp = [&](const uint32_t (&v)[32], int col0, int k0) {
+        if (masked) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, nsub));
+            float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, nsub));
+            p0 = (col0 + 2 * i < nvis) ? p0 : 0.f;
+            p1 = (col0 + 2 * i + 1 < nvis) ? p1 : 0.f;
+            rs0 += p0; rs1 += p1;
+            pk[k0 + i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float x0, x1, q0, q1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, ns2), x0, x1);
+            const uint64_t pp = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
+            if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
+            unpack_f32x2(mul_f32x2(pp, ps2), q0, q1);
+            pk[k0 + i] = pack_bf16x2(q0, q1);
+          }
+        }
+      };
+#pragma unroll 1
+      for (int h = 0; h < npages; ++h) {
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+        chunk_exp(b0, 64 * h, 0);
+        tmem_wait_ld();
+        if (h + 1 < npages) {
+          tmem_ld_32x32b_x32(scol + 64 * (h + 1), b0);
+        } else {                       // the score tile has been read for the last time
+          tc_fence_before_sync();
+          mbar_arrive(bar(A_SEMPTY + sb));
+          if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
+        }
+        chunk_exp(b1, 64 * h + 32, 16);
+        // stage P~ and N; the copy warps ship them to the value CTA
+        const uint32_t s2 = gt & 1;
+        if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
+        // one staging buffer: the copy warps of the previous page must have read it into registers
+        if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+        if (!ok) break;
+        if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
+        const uint32_t stg = smem_base + kOffStage;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        // the rescale (if any) belongs to the first half; the second half leaves O alone
+        const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
+                                            : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
+        st_shared_b32(stg + kPBytes + r * 4, nword);
+        mbar_arrive(bar(A_PSTAGED + s2));
+        if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
+        ++gt;
+      }
+      {
+        float s0, s1;
+        unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
+        rs0 += s0; rs1 += s1;
+      }
+      st.l = st.l * sp.l_up + (rs0 + rs1);
+    }
+    // line 20 scalars: 1 / (l * S16) and lse = m + ln l
+    if (ok) {
+      const bool live = st.l > 0.f;
+      const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
+      const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
+      const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;
+      st_cluster_b32(fdst, __float_as_uint(inv));
+      st_cluster_b32(fdst + 4, __float_as_uint(lse));
+      mbar_arrive_cluster(peerB_bars + 8u * (B_FINFULL + (un & 1)));
+    }
+  }
+  return (static_cast<uint64_t>(gt) << 32) | (static_cast<uint64_t>(gs) << 1) | (ok ? 1u : 0u);
+}
+
 }  // namespace
 
 template <int kMode, bool kGuard>
@@ -297,8 +452,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       // ---- softmax warpgroup: thread = query row
       const int r = tid;
       const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
-      const bool scale_nonneg = prm.scale_log2 >= 0.f;
-      const uint32_t mask_fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
+      const RoleCtx ctx{smem_base, bars, tbase, peerB_bars, peerB_base, prefix, seqlens, part, tid};
       while (ok && iter.next(u)) {
         // Q row -> tensor memory / shared memory (the previous unit's QK^T must be finished with it)
         ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
@@ -316,135 +470,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         tc_fence_before_sync();
         mbar_arrive(bar(A_QREADY));
         if (tid == 0) AMLA_STAMP(prm, part, 11, un);
-
-        RowState st;
-        row_state_init(st);
-        const int tok = (u.r0 + r) / prm.H;
-        const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);          // keys 0..visible-1 are seen by this row
-        const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // pages from here on may hold hidden keys
-
-        for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
-          const int npages = min(2, u.t1 - t);
-          const uint32_t sb = gs & 1;
-          ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
-          if (!ok) break;
-          tc_fence_after_sync();
-          if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
-          const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
-          const bool masked = t + npages > first_masked_tile;
-          const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
-
-          // The S tile is read from tensor memory in 32-column chunks, twice (maximum, then exponentials); the load
-          // of the next chunk is always in flight while a chunk is processed, so that the TMEM latency is hidden.
-          uint32_t b0[32], b1[32];
-          // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
-          float ext = scale_nonneg ? -INFINITY : INFINITY;
-          auto chunk_max = [&](uint32_t (&v)[32], int col0) {
-            if (masked) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) v[i] = (col0 + i < nvis) ? v[i] : mask_fill;
-            }
-            if (scale_nonneg) {
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) ext = fmax3(ext, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) ext = fminf(ext, fminf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
-            }
-          };
-          tmem_ld_32x32b_x32(scol, b0);
-#pragma unroll 1
-          for (int h = 0; h < npages; ++h) {
-            tmem_wait_ld();
-            tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
-            chunk_max(b0, 64 * h);
-            tmem_wait_ld();
-            tmem_ld_32x32b_x32(scol + (h + 1 < npages ? 64 * (h + 1) : 0), b0);   // next half, or the first chunk again for the second pass
-            chunk_max(b1, 64 * h + 32);
-          }
-          const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
-          const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
-          const float nsub = -sp.m2_sub;
-          float rs0 = 0.f, rs1 = 0.f;
-          const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
-          const uint64_t ps2 = pack_f32x2(sp.p_scale, sp.p_scale);
-          uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
-          uint32_t pk[32];
-          // lines 6, 10 for 32 columns: P, row sum (FP32, unscaled), P~ = bf16(P * S16), two elements per instruction
-          auto chunk_exp = [&](const uint32_t (&v)[32], int col0, int k0) {
-            if (masked) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, nsub));
-                float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, nsub));
-                p0 = (col0 + 2 * i < nvis) ? p0 : 0.f;
-                p1 = (col0 + 2 * i + 1 < nvis) ? p1 : 0.f;
-                rs0 += p0; rs1 += p1;
-                pk[k0 + i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
-              }
-            } else {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                float x0, x1, q0, q1;
-                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, ns2), x0, x1);
-                const uint64_t pp = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
-                if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
-                unpack_f32x2(mul_f32x2(pp, ps2), q0, q1);
-                pk[k0 + i] = pack_bf16x2(q0, q1);
-              }
-            }
-          };
-#pragma unroll 1
-          for (int h = 0; h < npages; ++h) {
-            tmem_wait_ld();
-            tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
-            chunk_exp(b0, 64 * h, 0);
-            tmem_wait_ld();
-            if (h + 1 < npages) {
-              tmem_ld_32x32b_x32(scol + 64 * (h + 1), b0);
-            } else {                       // the score tile has been read for the last time
-              tc_fence_before_sync();
-              mbar_arrive(bar(A_SEMPTY + sb));
-              if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
-            }
-            chunk_exp(b1, 64 * h + 32, 16);
-            // stage P~ and N; the copy warps ship them to the value CTA
-            const uint32_t s2 = gt & 1;
-            if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
-            // one staging buffer: the copy warps of the previous page must have read it into registers
-            if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
-            if (!ok) break;
-            if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
-            const uint32_t stg = smem_base + kOffStage;
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            // the rescale (if any) belongs to the first half; the second half leaves O alone
-            const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
-                                                : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
-            st_shared_b32(stg + kPBytes + r * 4, nword);
-            mbar_arrive(bar(A_PSTAGED + s2));
-            if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
-            ++gt;
-          }
-          {
-            float s0, s1;
-            unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
-            rs0 += s0; rs1 += s1;
-          }
-          st.l = st.l * sp.l_up + (rs0 + rs1);
-        }
-        if (!ok) break;
-        // line 20 scalars: 1 / (l * S16) and lse = m + ln l
-        {
-          const bool live = st.l > 0.f;
-          const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
-          const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
-          const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;
-          st_cluster_b32(fdst, __float_as_uint(inv));
-          st_cluster_b32(fdst + 4, __float_as_uint(lse));
-          mbar_arrive_cluster(peerB_bars + 8u * (B_FINFULL + (un & 1)));
-        }
+        // the unit's score tiles and its final scalars
+        const uint64_t ret = softmax_unit<kMode>(prm, ctx, u, un, gt, gs);
+        gt = static_cast<uint32_t>(ret >> 32);
+        gs = static_cast<uint32_t>(ret & 0xffffffffu) >> 1;
+        ok = (ret & 1u) != 0;
         ++un;
       }
       if (!ok) report_timeout(prm.status);
