@@ -22,6 +22,7 @@
 //
 // All waits are bounded; on expiry the kernel records kStatusTimeout and unwinds.
 #include <atomic>
+#include <type_traits>
 
 #include "amla_common.cuh"
 #include "amla_sm100.cuh"
@@ -221,25 +222,37 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
       tc_fence_after_sync();
       if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
       const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
-      const bool masked = t + npages > first_masked_tile;
       const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
+      // Two compilations of the tile: the plain one (every key visible, non-negative scale), and the general one
+      // with the visibility masks and the sign of the scale; a run-time flag inside one body costs the plain
+      // tiles their instruction schedule.
+      auto tile_body = [&](auto general_c) {
+      constexpr bool kGeneral = decltype(general_c)::value;
+      constexpr bool masked = kGeneral;
+      const bool scale_nn = kGeneral ? scale_nonneg : true;
 
       // The S tile is read from tensor memory in 32-column chunks, twice (maximum, then exponentials); the load
       // of the next chunk is always in flight while a chunk is processed, so that the TMEM latency is hidden.
       uint32_t b0[32], b1[32];
       // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
-      float ext = scale_nonneg ? -INFINITY : INFINITY;
+      float ext = scale_nn ? -INFINITY : INFINITY, ext_b = ext;      // two chains: half the dependent latency
       auto chunk_max = [&](uint32_t (&v)[32], int col0) {
         if (masked) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = (col0 + i < nvis) ? v[i] : mask_fill;
         }
-        if (scale_nonneg) {
+        if (scale_nn) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) ext = fmax3(ext, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+          for (int i = 0; i < 32; i += 4) {
+            ext = fmax3(ext, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            ext_b = fmax3(ext_b, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          }
         } else {
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) ext = fminf(ext, fminf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+          for (int i = 0; i < 32; i += 4) {
+            ext = fminf(ext, fminf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+            ext_b = fminf(ext_b, fminf(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3])));
+          }
         }
       };
       tmem_ld_32x32b_x32(scol, b0);
@@ -252,12 +265,15 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
         tmem_ld_32x32b_x32(scol + (h + 1 < npages ? 64 * (h + 1) : 0), b0);   // next half, or the first chunk again for the second pass
         chunk_max(b1, 64 * h + 32);
       }
+      ext = scale_nn ? fmaxf(ext, ext_b) : fminf(ext, ext_b);
       const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
       const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
-      const float nsub = -sp.m2_sub;
+      // Line 10's factor S16 goes into the exponential's argument (the paper's remark after Algorithm 2):
+      // P * S16 = 2^(a - m + log2 S16).  The row sum of line 6 is the sum of the same FP32 values, taken
+      // before the bf16 cast and divided by S16 once per tile.
+      const float nsub = log2f_approx(sp.p_scale) - sp.m2_sub;
       float rs0 = 0.f, rs1 = 0.f;
       const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
-      const uint64_t ps2 = pack_f32x2(sp.p_scale, sp.p_scale);
       uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
       uint32_t pk[32];
       // lines 6, 10 for 32 columns: P, row sum (FP32, unscaled), P~ = bf16(P * S16), two elements per instruction
@@ -270,16 +286,16 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
             p0 = (col0 + 2 * i < nvis) ? p0 : 0.f;
             p1 = (col0 + 2 * i + 1 < nvis) ? p1 : 0.f;
             rs0 += p0; rs1 += p1;
-            pk[k0 + i] = pack_bf16x2(p0 * sp.p_scale, p1 * sp.p_scale);
+            pk[k0 + i] = pack_bf16x2(p0, p1);
           }
         } else {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            float x0, x1, q0, q1;
+            float x0, x1;
             unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, ns2), x0, x1);
-            const uint64_t pp = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
+            const float q0 = ex2_approx(x0), q1 = ex2_approx(x1);
+            const uint64_t pp = pack_f32x2(q0, q1);
             if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
-            unpack_f32x2(mul_f32x2(pp, ps2), q0, q1);
             pk[k0 + i] = pack_bf16x2(q0, q1);
           }
         }
@@ -297,12 +313,15 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           mbar_arrive(bar(A_SEMPTY + sb));
           if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
         }
+        // One staging buffer: the copy warps of the previous page must have read it into registers.  The barrier is
+        // probed here, ahead of the last chunk's arithmetic, so that the probe's latency is not exposed (this warp
+        // is alone on its scheduler); the blocking wait runs only if the probe came too early.
+        const bool stage_free = gt == 0 || mbar_probe(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
         chunk_exp(b1, 64 * h + 32, 16);
         // stage P~ and N; the copy warps ship them to the value CTA
         const uint32_t s2 = gt & 1;
         if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
-        // one staging buffer: the copy warps of the previous page must have read it into registers
-        if (gt > 0) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+        if (!__all_sync(0xffffffffu, stage_free)) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
         if (!ok) break;
         if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
         const uint32_t stg = smem_base + kOffStage;
@@ -322,7 +341,10 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
         unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
         rs0 += s0; rs1 += s1;
       }
-      st.l = st.l * sp.l_up + (rs0 + rs1);
+      st.l = st.l * sp.l_up + __fdividef(rs0 + rs1, sp.p_scale);
+      };
+      if (t + npages > first_masked_tile || !scale_nonneg) tile_body(std::true_type{});
+      else tile_body(std::false_type{});
     }
     // line 20 scalars: 1 / (l * S16) and lse = m + ln l
     if (ok) {
@@ -606,11 +628,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         total *= 3;
         uint32_t par = 0;
         int g = lane;
+        int gs2 = lane & 1;                       // lanes 4..7: score tile whose SFULL (4, 5) / SEMPTY (6, 7) phase comes next
         const uint64_t t_start = global_timer_ns();
         for (uint32_t spin = 0;; ++spin) {
           const bool act = lane < kNumKSlots && g < total;
           if (act && mbar_probe(bar(A_KFULL + lane), par)) { AMLA_STAMP2(prm, part, 24, g); g += kNumKSlots; par ^= 1; }
-          if (!__any_sync(0xffffffffu, act)) break;
+          const bool act2 = lane >= 4 && lane < 8 && gs2 < total / 3;
+          if (act2 && mbar_probe(bar((lane < 6 ? A_SFULL : A_SEMPTY) + (lane & 1)), par)) { AMLA_STAMP2(prm, part, lane < 6 ? 30 : 31, gs2); gs2 += 2; par ^= 1; }
+          if (!__any_sync(0xffffffffu, act || act2)) break;
           if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) break;
         }
       }
