@@ -142,12 +142,14 @@ int amla_check_status(const void* workspace, void* cuda_stream);
 int amla_last_launch_count(void);
 
 /* Measurement aid (the one piece of per-thread state in the library): when enabled, every decode call
- * on this thread records CUDA events on its stream before and after each of its three launches
- * (schedule, decode, combine).  The events are created on the first enable and live until exit. */
+ * on this thread records CUDA events on its stream around its launches: before the schedule kernel
+ * (which only batches of more than 2048 items have; otherwise that interval is empty), between it and
+ * the decode kernel, between decode and combine, and after.  The events are created on the first
+ * enable and live until exit. */
 int amla_profile_enable(int on);
 
-/* Waits for the last profiled call on this thread and writes the elapsed milliseconds of its three
- * kernels (schedule, decode, combine) to ms3[0..2].  AMLA_ERR_INVALID_ARG if nothing was profiled. */
+/* Waits for the last profiled call on this thread and writes the elapsed milliseconds of the three
+ * intervals (schedule, decode, combine) to ms3[0..2].  AMLA_ERR_INVALID_ARG if nothing was profiled. */
 int amla_profile_last_ms(float* ms3);
 
 /*

@@ -133,7 +133,7 @@ cudaError_t launch_plan(const DecodeParams& prm, int* prefix_out, cudaStream_t s
 }
 
 cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream) {
-  const int warps_per_block = 8;
+  const int warps_per_block = 4;   // small blocks: one fits beside a decode CTA (registers), so part of the grid is resident before the decode kernel ends
   const long rows = static_cast<long>(prm.B) * prm.nrb * kRowBlock;
   const int blocks = static_cast<int>((rows + warps_per_block - 1) / warps_per_block);
   // programmatic dependent launch: the blocks may be placed while the decode kernel drains; they wait inside

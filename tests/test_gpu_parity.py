@@ -52,6 +52,15 @@ def test_many_short_sequences_more_items_than_parts():
     check_full(w)
 
 
+@pytest.mark.parametrize("B", [128, 129])
+def test_items_around_the_on_chip_schedule_copy(B):
+    # up to 128 items the CTAs keep the schedule prefix and the sequence lengths in shared memory, above they read them
+    # from the workspace
+    rng = np.random.default_rng(12 + B)
+    w = synth.make_workload("edge", B, 1, 16, rng.integers(0, 300, B), seed=13)
+    check_full(w)
+
+
 def test_more_items_than_the_in_kernel_schedule_handles():
     # above 2048 (sequence, row block) items the schedule prefix comes from its own kernel instead of the decode kernel
     rng = np.random.default_rng(10)
