@@ -160,3 +160,10 @@ def test_config4_rescale_stress_sampled():
 
 def test_config5_long_context_split_sampled():
     check_sampled(synth.config_long(), 64)
+
+
+def test_paper_grid_point_sampled():
+    # one point of the paper's own benchmark grid (Section 5.2: batch 96, S_q = 2, S_k = 1024): 192 work items
+    from paper_2509_25224_b200 import paper_grid
+    check_sampled(paper_grid.grid_workload(2, 1024), 128)
+
