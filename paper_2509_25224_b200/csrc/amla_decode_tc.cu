@@ -724,13 +724,30 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             if (!ok) break;
             tc_fence_after_sync();
             // two 32-column chunks in flight: the load of one overlaps the arithmetic of the other
+            // The guarded add costs four integer operations per element, the FP32 multiply it replaces one.  The guard
+            // only matters for an element whose magnitude bits plus N would not stay positive (an exact zero, a value
+            // about to leave the normal range); so the smallest magnitude of the chunk is taken first (half an
+            // operation per element), and where it is safe the chunk gets the plain one-instruction add of Lemma 3.1.
             auto apply = [&](uint32_t (&o)[32]) {
+              if (kMode == 2) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                float f = __uint_as_float(o[i]);
-                if (kMode == 2) f *= __uint_as_float(nword);
-                else f = kGuard ? exponent_add_guarded(f, static_cast<int>(nword)) : exponent_add_raw(f, static_cast<int>(nword));
-                o[i] = __float_as_uint(f);
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * __uint_as_float(nword));
+              } else if (!kGuard) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(exponent_add_raw(__uint_as_float(o[i]), static_cast<int>(nword)));
+              } else {
+                float lo = fmin3_abs(__uint_as_float(o[0]), __uint_as_float(o[1]), __uint_as_float(o[2]));
+#pragma unroll
+                for (int i = 3; i + 1 < 32; i += 2) lo = fmin3_abs(lo, __uint_as_float(o[i]), __uint_as_float(o[i + 1]));
+                lo = fminf(lo, fabsf(__uint_as_float(o[31])));
+                // NaN magnitudes compare as large numbers and take the plain add, like every other normal pattern
+                if (__float_as_int(lo) + static_cast<int>(nword) > 0) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(exponent_add_raw(__uint_as_float(o[i]), static_cast<int>(nword)));
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(exponent_add_guarded(__uint_as_float(o[i]), static_cast<int>(nword)));
+                }
               }
             };
             uint32_t o0[32], o1[32];
