@@ -395,7 +395,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       mbar_init(bar(A_QFREE), 1);
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
-      for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 128); }
+      for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 256); }
       for (int i = 0; i < 2; ++i) mbar_init(bar(B_FINFULL + i), 128);
     }
     fence_mbar_init();
@@ -705,10 +705,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   } else {
     // ======================================================================= value CTA
     uint32_t gv = 0;    // V ring slots so far (two per page)
-    if (wid < 4) {
-      // ---- correction + epilogue warpgroup: thread = query row
-      const int r = tid;
-      const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+    if (wid < 4 || (wid >= 6 && wid < 10)) {
+      // ---- correction + epilogue warpgroup: thread = query row.  A warp reaches the tensor-memory lanes
+      // 32 * (warp % 4) .. + 31, so warps 6-9, which have no other work in this CTA, are the partners of warps 2, 3,
+      // 0, 1: each of a pair rescales one half of the row's 512 columns.  The epilogue stays with warps 0-3.
+      const bool partner = wid >= 4;
+      const int r = (wid & 3) * 32 + lane;
+      const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+      const int c_first = partner ? 8 : 0;          // first of this warp's eight 32-column chunks
       while (ok && iter.next(u)) {
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
           const uint32_t s = gt % kNumP, k = gt / kNumP;
@@ -751,16 +755,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
               }
             };
             uint32_t o0[32], o1[32];
-            const uint32_t obase = tbase + lane_base;
+            const uint32_t obase = tbase + lane_base + 32 * c_first;
             tmem_ld_32x32b_x32(obase, o0);
 #pragma unroll 1
-            for (int c = 0; c < 16; c += 2) {
+            for (int c = 0; c < 8; c += 2) {
               tmem_wait_ld();
               tmem_ld_32x32b_x32(obase + 32 * (c + 1), o1);
               apply(o0);
               tmem_st_32x32b_x32(obase + 32 * c, o0);
               tmem_wait_ld();
-              if (c + 2 < 16) tmem_ld_32x32b_x32(obase + 32 * (c + 2), o0);
+              if (c + 2 < 8) tmem_ld_32x32b_x32(obase + 32 * (c + 2), o0);
               apply(o1);
               tmem_st_32x32b_x32(obase + 32 * (c + 1), o1);
             }
@@ -772,7 +776,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         }
         if (!ok) break;
         // ---- epilogue (line 20): out = O / (l * S16)
-        {
+        if (!partner) {
           const uint32_t gl = gt - 1;
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
