@@ -167,3 +167,29 @@ def test_paper_grid_point_sampled():
     from paper_2509_25224_b200 import paper_grid
     check_sampled(paper_grid.grid_workload(2, 1024), 128)
 
+
+def test_rescale_mode_accuracy_table(capsys):
+    # Accuracy of the three ways to rescale O (Algorithm 2's integer add, Eq. 3's exact fold, Algorithm 1's FP32
+    # multiply), each with the reference moved at every new maximum (tau = 0) and lazily (tau = 8), against the FP64
+    # oracle: the paper's claim (Tables 3-4) is that the integer add costs no accuracy against the multiply.
+    cases = [("staircase B=2 N=4096", synth.config_stress(B=2, N=4096)),
+             ("normal    B=2 N=8192", synth.make_workload("n", 2, 1, 128, [8192, 8192], seed=77))]
+    modes = [("alg2", binding.RESCALE_ALG2), ("fold", binding.RESCALE_FOLD), ("fmul", binding.RESCALE_FMUL)]
+    lines = []
+    for name, w in cases:
+        ro, rl = R.decode(w.q, w.kv, w.block_table, w.seqlens, w.scale)
+        dev = to_device(w)
+        rel = {}
+        for mn, mf in modes:
+            for tau in (0, 8):
+                out, lse, _ = run_gpu(w, mf | binding.lazy(tau), dev_inputs=dev)
+                err = float(np.abs(out - ro).max())
+                rel[mn, tau] = float(np.linalg.norm(out - ro) / np.linalg.norm(ro))
+                le = float(np.abs(lse - rl).max())
+                lines.append(f"{name} {mn:5s} tau={tau}: max|err| {err:.3e} rel_l2 {rel[mn, tau]:.3e} lse_err {le:.2e}")
+                assert err <= 2e-2 and rel[mn, tau] <= 5e-3 and le <= 1e-3
+        for tau in (0, 8):   # the integer add stays within 10 % of the multiply's error
+            assert rel["alg2", tau] <= 1.10 * rel["fmul", tau]
+    with capsys.disabled():
+        print("\n" + "\n".join(lines))
+
