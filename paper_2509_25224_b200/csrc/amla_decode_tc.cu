@@ -704,7 +704,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     }
   } else {
     // ======================================================================= value CTA
-    uint32_t gv = 0;    // V ring slots so far (two per page)
     if (wid < 4 || (wid >= 6 && wid < 10)) {
       // ---- correction + epilogue warpgroup: thread = query row.  A warp reaches the tensor-memory lanes
       // 32 * (warp % 4) .. + 31, so warps 6-9, which have no other work in this CTA, are the partners of warps 2, 3,
