@@ -55,7 +55,10 @@ enum {
   AMLA_RESCALE_FMUL = 2,
   AMLA_RESCALE_MASK = 3,
   AMLA_FLAG_UNGUARDED_ADD = 4,
-  AMLA_FLAG_KERNEL_SIMT = 8,    /* run the scalar bring-up kernel instead of the tensor-core kernel */
+  AMLA_FLAG_KERNEL_SIMT = 8,    /* run the scalar bring-up kernel instead of the tensor-core kernels */
+  AMLA_FLAG_KERNEL_ROWS128 = 16, /* A/B measurements: treat sequences with more than 128 query rows as independent
+                                    128-row blocks (each streams the cache on its own) instead of running the
+                                    256-row kernel, in which one load of a cache tile serves all 256 rows */
   AMLA_LAZY_SHIFT = 8,
   AMLA_LAZY_MASK = 0xF00,
   AMLA_DEFAULT_TAU = 8
@@ -90,8 +93,9 @@ int amla_mla_decode_workspace_size(int B, int Sq, int H, int max_blocks_per_seq,
  *                need not be preserved or initialised; calls that overlap in time need distinct ones
  *   cuda_stream  a cudaStream_t (NULL = default stream)
  *
- * Supported: 1 <= Sq <= 8, 1 <= H <= 128 (any Sq*H up to 1024 query rows per sequence; rows are
- * processed in blocks of 128); page size 64; sm_100 devices only (AMLA_ERR_UNSUPPORTED otherwise).
+ * Supported: 1 <= Sq <= 8, 1 <= H <= 128 (any Sq*H up to 1024 query rows per sequence; up to 128 rows are
+ * processed as one block by a pair of SMs, more than 128 rows in blocks of 256 by four SMs that share every
+ * cache tile they load); page size 64; sm_100 devices only (AMLA_ERR_UNSUPPORTED otherwise).
  * Argument errors are reported before anything is launched.
  */
 int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_table,
@@ -119,13 +123,18 @@ int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_ta
  * it keeps the previous call's contents: that is harmless, because each call rewrites everything it later reads,
  * but two calls whose kernels overlap on the GPU (different streams, no ordering between them) race on it and
  * give undefined results.  Order such calls, or use amla_mla_decode with one workspace per stream.
- * The bounded-wait status word is inside the array; amla_check_status does not apply to this entry point.
+ * The bounded-wait status word is inside the array: read it with amla_static_check_status, not amla_check_status.
  */
 #define AMLA_STATIC_MAX_ITEMS 4096
 #define AMLA_STATIC_MAX_SMS 148
 int amla_mla_decode_static(const void* q, const void* kv_cache, const int32_t* block_table,
                            const int32_t* seqlens, float softmax_scale, int B, int Sq, int H, int num_blocks,
                            int max_blocks_per_seq, void* out, float* lse, void* cuda_stream);
+
+/* amla_check_status for amla_mla_decode_static: synchronises `cuda_stream` and reads the status word that the
+ * kernels keep in the built-in scratch of the current device.  AMLA_OK, or AMLA_ERR_DEVICE_TIMEOUT if a bounded
+ * wait expired during the last static call (its outputs are then undefined).  Allocates nothing. */
+int amla_static_check_status(void* cuda_stream);
 
 /* Same as amla_mla_decode, with a flags word selecting a rescale variant (see the enum above). */
 int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block_table,
@@ -137,6 +146,26 @@ int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block
  * workspace: AMLA_OK, or AMLA_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel expired (the
  * kernel then returned early and the outputs are undefined).  Optional. */
 int amla_check_status(const void* workspace, void* cuda_stream);
+
+/*
+ * Diagnostic: shows that a bounded device-side wait reports instead of hanging.  Launches a one-warp kernel that
+ * waits, with the wait routine of the decode kernels and a limit of `limit_ns` nanoseconds (1 .. 100 000 000),
+ * on a barrier nothing arrives on; when the limit passes it stores the time-out status in the first word of
+ * `workspace` (device, 4-byte aligned, at least 4 bytes) and ends.  amla_check_status(workspace, stream) then
+ * returns AMLA_ERR_DEVICE_TIMEOUT; the next decode call on that workspace resets the word.  No decode work runs.
+ */
+int amla_wait_selftest(void* workspace, unsigned long long limit_ns, void* cuda_stream);
+
+/*
+ * Debug aid, host only: checks HOST copies of the paging inputs before a decode call.  Every seqlens[b] must lie
+ * in [0, 64 * max_blocks_per_seq] and every block_table entry that the sequence uses (the first
+ * ceil(seqlens[b] / 64) of row b) in [0, num_blocks).  Returns AMLA_OK, or AMLA_ERR_INVALID_ARG with the
+ * offending sequence in *bad_seq and entry index in *bad_block (-1 when the length itself is out of range);
+ * either pointer may be NULL.  (The kernels never fault on a bad page index -- an out-of-range TMA coordinate
+ * reads as zeros -- so such a mistake shows up as wrong results only; this check names it.)  Nothing is launched.
+ */
+int amla_validate_paging_host(const int32_t* block_table, const int32_t* seqlens, int B, int num_blocks,
+                              int max_blocks_per_seq, int* bad_seq, int* bad_block);
 
 /* Number of kernels the most recent amla_mla_decode[_ex] call on this thread launched. */
 int amla_last_launch_count(void);
@@ -154,9 +183,11 @@ int amla_profile_last_ms(float* ms3);
 
 /*
  * Host mirror of the device-side split-KV schedule (the plan is not in the paper; it exists because
- * B * ceil(Sq*H/128) work items are far fewer than the SMs).  Items are (sequence, 128-row block)
- * pairs in order; their 64-key tiles, each non-empty item preceded by 10 overhead positions that stand
- * for the cost of starting an item, form one linear range that is cut into num_parts equal parts.
+ * B * ceil(Sq*H/128) work items are far fewer than the SMs).  For Sq*H <= 128 the items are (sequence, 128-row
+ * block) pairs, their tiles 64-key pages, and every non-empty item but the first is preceded by 10 overhead
+ * positions that stand for the cost of starting an item; for Sq*H > 128 the items are (sequence, 256-row block)
+ * pairs, the tiles 128 keys (two pages) and the overhead 5 positions.  Items in order form one linear range
+ * that is cut into num_parts equal parts.
  * For every (part, item) intersection ("unit") one record of 6 int32 is written:
  *   part, item, tile_begin, tile_end (within the item), slot (-1 = writes out/lse directly,
  *   otherwise index of its fp32 partial), n_split of the item.

@@ -20,6 +20,7 @@ RESCALE_FOLD = 1
 RESCALE_FMUL = 2
 FLAG_UNGUARDED_ADD = 4
 FLAG_KERNEL_SIMT = 8
+FLAG_KERNEL_ROWS128 = 16
 DEFAULT_TAU = 8
 
 
@@ -35,7 +36,8 @@ DEFAULT_FLAGS = RESCALE_ALG2 | lazy(DEFAULT_TAU)   # what amla_mla_decode (witho
 EXPORTS = [
     "amla_status_string", "amla_mla_decode_workspace_size", "amla_mla_decode", "amla_mla_decode_ex",
     "amla_check_status", "amla_last_launch_count", "amla_plan_host", "amla_profile_enable",
-    "amla_profile_last_ms", "amla_mla_decode_static",
+    "amla_profile_last_ms", "amla_mla_decode_static", "amla_static_check_status", "amla_wait_selftest",
+    "amla_validate_paging_host",
 ]
 
 _lib = None
@@ -67,6 +69,12 @@ def lib() -> ctypes.CDLL:
         L.amla_mla_decode_ex.restype = i32
         L.amla_mla_decode_static.argtypes = [vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, vp, vp, vp]
         L.amla_mla_decode_static.restype = i32
+        L.amla_static_check_status.argtypes = [vp]
+        L.amla_static_check_status.restype = i32
+        L.amla_wait_selftest.argtypes = [vp, ctypes.c_ulonglong, vp]
+        L.amla_wait_selftest.restype = i32
+        L.amla_validate_paging_host.argtypes = [vp, vp, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.amla_validate_paging_host.restype = i32
         L.amla_check_status.argtypes = [vp, vp]
         L.amla_check_status.restype = i32
         L.amla_last_launch_count.argtypes = []
@@ -95,7 +103,8 @@ def workspace_size(B: int, Sq: int, H: int, max_blocks_per_seq: int, device: int
 
 def plan_host(seqlens, Sq: int, H: int, num_parts: int) -> np.ndarray:
     """Host mirror of the split-KV schedule: int32 [n_units, 6] rows of
-    (part, item, tile_begin, tile_end, slot, n_split)."""
+    (part, item, tile_begin, tile_end, slot, n_split).  Items are 128-row blocks with 64-key tiles for
+    Sq*H <= 128, 256-row blocks with 128-key tiles above."""
     sl = np.ascontiguousarray(seqlens, dtype=np.int32)
     B = sl.shape[0]
     nrb = (Sq * H + 127) // 128
@@ -136,6 +145,36 @@ def mla_decode_static(q, kv_cache, block_table, seqlens, softmax_scale: float, o
                                           out.data_ptr(), lse.data_ptr(), stream)
     if rc != AMLA_OK:
         raise AmlaError(rc, "amla_mla_decode_static")
+
+
+def static_check_status(stream: int = 0) -> None:
+    """Raises AmlaError(-5) if a bounded wait expired during the last amla_mla_decode_static call on this device."""
+    rc = lib().amla_static_check_status(stream)
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_static_check_status")
+
+
+def wait_selftest(workspace, limit_ns: int = 1_000_000, stream: int = 0) -> None:
+    """Launches the bounded-wait self-test (a wait nothing satisfies, given up after limit_ns); afterwards
+    check_status(workspace) raises AmlaError(-5)."""
+    rc = lib().amla_wait_selftest(workspace.data_ptr(), int(limit_ns), stream)
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_wait_selftest")
+
+
+def validate_paging_host(block_table, seqlens, num_blocks: int):
+    """Host-side debug check of numpy copies of the paging inputs.  Returns None when they are consistent, else
+    (bad_seq, bad_block) with bad_block = -1 for an out-of-range length."""
+    bt = np.ascontiguousarray(block_table, dtype=np.int32)
+    sl = np.ascontiguousarray(seqlens, dtype=np.int32)
+    bs, bb = ctypes.c_int(-1), ctypes.c_int(-1)
+    rc = lib().amla_validate_paging_host(bt.ctypes.data_as(ctypes.c_void_p), sl.ctypes.data_as(ctypes.c_void_p),
+                                         bt.shape[0], int(num_blocks), bt.shape[1], ctypes.byref(bs), ctypes.byref(bb))
+    if rc == AMLA_OK:
+        return None
+    if rc != -1:
+        raise AmlaError(rc, "amla_validate_paging_host")
+    return int(bs.value), int(bb.value)
 
 
 def last_launch_count() -> int:

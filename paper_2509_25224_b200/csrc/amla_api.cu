@@ -2,6 +2,7 @@
 // (schedule prefix, decode, combine) on the caller's stream.
 #include <atomic>
 #include <cstring>
+#include <new>
 
 #include "../../include/amla.h"
 #include "amla_common.cuh"
@@ -12,7 +13,10 @@ cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream);
 cudaError_t launch_decode_simt(const DecodeParams& prm, cudaStream_t stream);
 // Returns cudaSuccess, or an error; sets *unsupported when the device cannot run the kernel.
 cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* unsupported);
+cudaError_t launch_decode_quad(const DecodeParams& prm, cudaStream_t stream, int* unsupported);
+cudaError_t launch_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t stream);
 int decode_tc_parts(int sm_count);
+int decode_quad_parts(int device, int sm_count);
 
 namespace {
 
@@ -81,6 +85,56 @@ void profile_mark(int i, cudaStream_t stream) {
 }
 
 }  // namespace
+
+// Chooses the kernel for the shape and fills the schedule fields of prm (rows per item, keys per tile, parts).
+// Sequences with more than 128 query rows go to the 256-row kernel (four-CTA clusters, pair MMAs) unless
+// AMLA_FLAG_KERNEL_ROWS128 asks for the 128-row kernel.
+int configure_schedule(DecodeParams& prm, int device, int sms, int flags) {
+  const bool simt = (flags & AMLA_FLAG_KERNEL_SIMT) != 0;
+  bool quad = !simt && !(flags & AMLA_FLAG_KERNEL_ROWS128) && prm.R > kRowBlock;
+  int quad_parts = 0;
+  if (quad) {
+    quad_parts = decode_quad_parts(device, sms);
+    if (quad_parts <= 0) quad = false;         // four-CTA clusters cannot be placed on this device
+  }
+  prm.item_rows = quad ? 2 * kRowBlock : kRowBlock;
+  prm.tile_keys = quad ? 2 * kPage : kPage;
+  prm.ovh = quad ? kUnitOverheadTiles / 2 : kUnitOverheadTiles;
+  prm.nrb = (prm.R + prm.item_rows - 1) / prm.item_rows;
+  prm.n_items = prm.B * prm.nrb;
+  prm.P = simt ? sms : quad ? quad_parts : decode_tc_parts(sms);
+  prm.fused_plan = (!simt && prm.n_items <= kFusedPlanMaxItems) ? 1 : 0;
+  return AMLA_OK;
+}
+
+// The launches of one decode call (schedule kernel for large batches, decode, combine) on `stream`.
+int launch_decode_call(const DecodeParams& prm, int* prefix, cudaStream_t stream, int* launches, void (*mark)(int, cudaStream_t)) {
+  const bool simt = (prm.flags & AMLA_FLAG_KERNEL_SIMT) != 0;
+  if (mark) mark(0, stream);
+  if (!prm.fused_plan) {
+    if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+    ++*launches;
+  }
+  if (mark) mark(1, stream);
+  if (simt) {
+    if (launch_decode_simt(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  } else {
+    int unsupported = 0;
+    const cudaError_t err = prm.item_rows > kRowBlock ? launch_decode_quad(prm, stream, &unsupported)
+                                                      : launch_decode_tc(prm, stream, &unsupported);
+    if (err != cudaSuccess) {
+      cudaGetLastError();
+      return unsupported ? AMLA_ERR_UNSUPPORTED : AMLA_ERR_CUDA;
+    }
+  }
+  ++*launches;
+  if (mark) mark(2, stream);
+  if (launch_combine(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  ++*launches;
+  if (mark) mark(3, stream);
+  return AMLA_OK;
+}
+
 }  // namespace amla
 
 using namespace amla;
@@ -134,9 +188,8 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   if (rc != AMLA_OK) return rc;
   if (cc != 10) return AMLA_ERR_UNSUPPORTED;
 
-  const int nrb = (Sq * H + kRowBlock - 1) / kRowBlock;
-  const int n_items = B * nrb;
-  const Layout lay = make_layout(n_items, sms);
+  // the layout is sized for 128-row items (the larger item count) whichever kernel runs
+  const Layout lay = make_layout(B * ((Sq * H + kRowBlock - 1) / kRowBlock), sms);
   if (workspace_bytes < lay.total) return AMLA_ERR_WORKSPACE;
 
   char* ws = static_cast<char*>(workspace);
@@ -156,8 +209,6 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   prm.scale_log2 = softmax_scale * kLog2e;
   prm.B = B; prm.Sq = Sq; prm.H = H;
   prm.R = Sq * H;
-  prm.nrb = nrb;
-  prm.n_items = n_items;
   prm.num_blocks = num_blocks;
   prm.max_blocks_per_seq = max_blocks_per_seq;
   prm.flags = flags;
@@ -165,33 +216,9 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   prm.trace = g_trace;
 #endif
   prm.tau = static_cast<float>((flags & AMLA_LAZY_MASK) >> AMLA_LAZY_SHIFT);
-  const bool simt = (flags & AMLA_FLAG_KERNEL_SIMT) != 0;
-  prm.P = simt ? sms : decode_tc_parts(sms);
-
-  prm.fused_plan = (!simt && n_items <= kFusedPlanMaxItems) ? 1 : 0;
-
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  profile_mark(0, stream);
-  if (!prm.fused_plan) {
-    if (launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-    ++g_last_launches;
-  }
-  profile_mark(1, stream);
-  if (simt) {
-    if (launch_decode_simt(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-  } else {
-    int unsupported = 0;
-    if (launch_decode_tc(prm, stream, &unsupported) != cudaSuccess) {
-      cudaGetLastError();
-      return unsupported ? AMLA_ERR_UNSUPPORTED : AMLA_ERR_CUDA;
-    }
-  }
-  ++g_last_launches;
-  profile_mark(2, stream);
-  if (launch_combine(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-  ++g_last_launches;
-  profile_mark(3, stream);
-  return AMLA_OK;
+  rc = configure_schedule(prm, device, sms, flags);
+  if (rc != AMLA_OK) return rc;
+  return launch_decode_call(prm, prefix, static_cast<cudaStream_t>(cuda_stream), &g_last_launches, profile_mark);
 }
 
 extern "C" int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_table,
@@ -216,6 +243,39 @@ extern "C" int amla_check_status(const void* workspace, void* cuda_stream) {
 }
 
 extern "C" int amla_last_launch_count(void) { return g_last_launches; }
+
+extern "C" int amla_wait_selftest(void* workspace, unsigned long long limit_ns, void* cuda_stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 3)) return AMLA_ERR_INVALID_ARG;
+  if (limit_ns == 0 || limit_ns > 100000000ull) return AMLA_ERR_INVALID_ARG;      // at most 0.1 s
+  if (launch_wait_selftest(static_cast<int*>(workspace), limit_ns, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return AMLA_ERR_CUDA;
+  }
+  return AMLA_OK;
+}
+
+extern "C" int amla_validate_paging_host(const int32_t* block_table, const int32_t* seqlens, int B, int num_blocks,
+                                         int max_blocks_per_seq, int* bad_seq, int* bad_block) {
+  if (!block_table || !seqlens || B <= 0 || num_blocks <= 0 || max_blocks_per_seq <= 0) return AMLA_ERR_INVALID_ARG;
+  for (int b = 0; b < B; ++b) {
+    const long long n = seqlens[b];
+    if (n < 0 || n > static_cast<long long>(max_blocks_per_seq) * kPage) {
+      if (bad_seq) *bad_seq = b;
+      if (bad_block) *bad_block = -1;
+      return AMLA_ERR_INVALID_ARG;
+    }
+    const int used = static_cast<int>((n + kPage - 1) / kPage);
+    for (int i = 0; i < used; ++i) {
+      const int32_t pg = block_table[static_cast<size_t>(b) * max_blocks_per_seq + i];
+      if (pg < 0 || pg >= num_blocks) {
+        if (bad_seq) *bad_seq = b;
+        if (bad_block) *bad_block = i;
+        return AMLA_ERR_INVALID_ARG;
+      }
+    }
+  }
+  return AMLA_OK;
+}
 
 extern "C" int amla_profile_enable(int on) {
   if (on && !g_ev[0]) {
@@ -243,16 +303,20 @@ extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int 
   if (!seqlens || !units || num_parts <= 0 || max_units < 0) return AMLA_ERR_INVALID_ARG;
   int rc = check_shape(B, Sq, H, 1);
   if (rc != AMLA_OK) return rc;
-  const int nrb = (Sq * H + kRowBlock - 1) / kRowBlock;
+  const bool quad = Sq * H > kRowBlock;
+  const int item_rows = quad ? 2 * kRowBlock : kRowBlock, tile_keys = quad ? 2 * kPage : kPage;
+  const int ovh = quad ? kUnitOverheadTiles / 2 : kUnitOverheadTiles;
+  const int nrb = (Sq * H + item_rows - 1) / item_rows;
   const int n_items = B * nrb;
-  int* prefix = new int[n_items + 1];
+  int* prefix = new (std::nothrow) int[n_items + 1];
+  if (!prefix) return AMLA_ERR_WORKSPACE;
   int acc = 0;
   for (int it = 0; it < n_items; ++it) {
     prefix[it] = acc;
-    acc += schedule_length(seqlens[it / nrb], it);
+    acc += schedule_length(seqlens[it / nrb], it, tile_keys, ovh);
   }
   prefix[n_items] = acc;
-  const Plan plan = Plan::make(prefix, n_items, num_parts);
+  const Plan plan = Plan::make(prefix, n_items, num_parts, ovh);
   int n_units = 0;
   bool overflow = false;
   if (acc > 0) {

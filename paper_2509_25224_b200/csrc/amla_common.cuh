@@ -40,6 +40,9 @@ struct DecodeParams {
   int P;                         // parts the linear tile range is cut into
   int fused_plan;                // the decode kernel computes `prefix` itself (few items), no schedule kernel
   int flags;
+  int tile_keys;                 // keys per schedule tile: 64 (one page) or 128 (two pages, the 256-row kernel)
+  int item_rows;                 // query rows per work item: 128, or 256 for the 256-row kernel (nrb counts these)
+  int ovh;                       // schedule positions that stand for the cost of starting an item
   unsigned long long* trace;     // timeline buffer of a -DAMLA_TRACE build, else unused (nullptr)
 };
 
@@ -66,24 +69,24 @@ constexpr int kTraceTiles = 96;
 
 // ---------------------------------------------------------------------------------------------
 // Split-KV schedule.  Items (sequence b, row block rb) in order it = b * nrb + rb own
-// ceil(N_b / 64) tiles each.  Starting an item costs a cluster a fixed amount of time (its Q rows,
+// ceil(N_b / tile_keys) tiles each (a tile is one 64-key page for the 128-row kernel, two for the 256-row one).  Starting an item costs a cluster a fixed amount of time (its Q rows,
 // the pipeline fill, the epilogue) that is worth about kUnitOverheadTiles tiles, so the schedule
 // balances a linear range in which every non-empty item but the first is preceded by that many
 // overhead positions: prefix[it] is the position where item `it` begins (overhead first, then its tiles),
 // L = prefix[n_items] the total, and part p owns positions [p*L/P, (p+1)*L/P).  A part does the
 // tiles whose positions it owns; overhead positions carry no work.
 // ---------------------------------------------------------------------------------------------
-constexpr int kUnitOverheadTiles = 10;
+constexpr int kUnitOverheadTiles = 10;        // in 64-key pages; halved when tiles are 128 keys
 constexpr int kFusedPlanMaxItems = 2048;   // up to this many items every decode CTA computes the prefix itself
 
 // Overhead positions in front of item `it`: none for the first item, which opens the first part anyway (every
 // part pays for one start; the positions stand for the additional ones).
-__host__ __device__ inline int item_overhead(int it) { return it > 0 ? kUnitOverheadTiles : 0; }
+__host__ __device__ inline int item_overhead(int it, int ovh) { return it > 0 ? ovh : 0; }
 // Schedule length of an item: its tiles plus the start-up overhead (nothing for an empty sequence).
-__host__ __device__ inline int schedule_length(int seqlen, int it) {
+__host__ __device__ inline int schedule_length(int seqlen, int it, int tile_keys, int ovh) {
   const int n = seqlen < 0 ? 0 : seqlen;
-  const int tiles = (n + kPage - 1) / kPage;
-  return tiles > 0 ? tiles + item_overhead(it) : 0;
+  const int tiles = (n + tile_keys - 1) / tile_keys;
+  return tiles > 0 ? tiles + item_overhead(it, ovh) : 0;
 }
 
 struct Plan {
@@ -91,12 +94,14 @@ struct Plan {
   int n_items;
   int L;
   int P;
+  int ovh;
   bool wide;     // L * P does not fit 31 bits: the part arithmetic needs 64-bit division (slow on the device)
 
   // With fewer positions than parts only the first L parts exist (one position each).
-  __host__ __device__ static Plan make(const int* prefix, int n_items, int max_parts) {
+  __host__ __device__ static Plan make(const int* prefix, int n_items, int max_parts, int ovh) {
     Plan pl;
     pl.prefix = prefix;
+    pl.ovh = ovh;
     pl.n_items = n_items;
     pl.L = prefix[n_items];
     pl.P = pl.L < max_parts ? (pl.L > 0 ? pl.L : 1) : max_parts;
@@ -129,7 +134,7 @@ struct Plan {
     return lo;
   }
   // Position of the first tile of a non-empty item.
-  __host__ __device__ int first_tile(int it) const { return prefix[it] + item_overhead(it); }
+  __host__ __device__ int first_tile(int it) const { return prefix[it] + item_overhead(it, ovh); }
   // Parts [p_first, p_last] that hold tiles of item `it`; returns the split count (0 for an empty item).
   __host__ __device__ int item_parts(int it, int* p_first, int* p_last) const {
     const int e = prefix[it + 1];

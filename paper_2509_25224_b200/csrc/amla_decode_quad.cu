@@ -1,0 +1,972 @@
+// Tensor-core MLA decode kernel for sequences with more than 128 query rows (S_q >= 2 with 128 heads), sm_100a.
+//
+// A cluster of four CTAs works on one block of 256 query rows and a range of 128-key tiles (two cache pages):
+//
+//   score pair (cluster ranks 0, 1)   CTA j keeps rows 128 j .. 128 j + 127 of Q (latent part in tensor memory, RoPE
+//       part in shared memory) and loads ONE page of every tile: S = Q K^T is a pair MMA (M = 256, N = 128, K = 16,
+//       issued by rank 0) whose B operand is split over the two CTAs, so that every key row enters the shared
+//       memory of one SM only and serves all 256 query rows.  Each CTA runs the softmax of its own 128 rows
+//       (Algorithm 2's per-row recurrence, lines 5-12) and ships P~ = bf16(P * S16) and the per-row integers N to
+//       "its" value CTA.
+//   value pair (cluster ranks 2, 3)   CTA j holds the FP32 accumulator O of rows 128 j .. in its tensor memory; the
+//       P~ V product is a pair MMA (M = 256, N = 256) whose B operand (V: 128 of the 256 columns per CTA) is again
+//       split, so each value CTA loads half of every V tile.  The correction warps apply N to the bit patterns of O
+//       (lines 13-16; Lemma 3.1); the epilogue divides by l * S16 (line 20).
+//
+// The roles, their rings and the order [QK^T(i+1), P~V(i), softmax(i+1)] (the paper's [C1, C2, V1] steady state,
+// Section 4.1) are those of the 128-row kernel; what changes is that the operand traffic per SM and key is halved,
+// which is what bounds that kernel.  Loads are plain TMA tile loads of each CTA into its own shared memory (no
+// multicast); the bytes of both halves are counted on one barrier of the pair's even CTA.
+//
+// All waits are bounded; on expiry the kernel records kStatusTimeout and unwinds.
+#include <atomic>
+#include <type_traits>
+
+#include "amla_common.cuh"
+#include "amla_sm100.cuh"
+
+namespace amla {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kNumCopyWarps = 4;
+constexpr int kThreads = 32 * (6 + kNumCopyWarps);   // warps 0-3: softmax / correction, 4: TMA producers, 5: MMA issuer + TMEM alloc, 6-9: P copy / correction partners
+constexpr int kTileKeys = 2 * kPage;                 // keys per schedule tile
+constexpr int kItemRows = 2 * kRowBlock;             // query rows per work item
+constexpr uint32_t kBoxBytes = 64 * 64 * 2;          // one 64-key x 64-column TMA box
+constexpr uint32_t kPBytes = 128 * 64 * 2;           // P~ of one page: 128 rows x 128 B
+constexpr uint32_t kNOff = kPBytes;                  // ... followed by the 128 per-row integers
+constexpr uint32_t kFinOff = kPBytes + 128 * 4;      // ... and, with a unit's last page, 128 x (1/(l*S16), lse)
+constexpr uint32_t kPXfer = kFinOff;
+constexpr uint32_t kPXferLast = kFinOff + 128 * 8;
+constexpr uint32_t kPStride = 18 * 1024;
+constexpr int kNumP = 4;                             // P buffers in a value CTA (pages the softmax may run ahead)
+
+// ---- score CTA
+constexpr int kNumKSlots = 6;                        // two tiles in flight per CTA
+constexpr uint32_t kKSlotBytes = 3 * kBoxBytes;      // 64 keys x 192 columns: [8 row groups][3 blocks][8 rows][128 B]
+constexpr uint32_t kKGroupStride = 3 * 1024;
+constexpr uint32_t kOffQRope = 0;                    // 128 rows x 64 bf16, 128-byte swizzle
+constexpr uint32_t kOffStage = 128 * 64 * 2;         // one staged page (P~, N, final scalars)
+constexpr uint32_t kOffK = kOffStage + kPStride;
+constexpr uint32_t kEndA = kOffK + kNumKSlots * kKSlotBytes;
+// ---- value CTA
+constexpr int kNumVSlots = 4;
+constexpr uint32_t kVHalfBytes = 2 * kBoxBytes;      // 64 keys x 128 columns: [2 blocks][64 keys][128 B]
+constexpr uint32_t kVSlotBytes = 2 * kVHalfBytes;    // one page: this CTA's 128 columns of either 256-column half of V
+constexpr uint32_t kOffV = 0;
+constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;
+constexpr uint32_t kOffEpi = kOffP + kNumP * kPStride;
+constexpr uint32_t kEndB = kOffEpi + 4 * 32 * 128;
+// ---- all four: barriers at the same offset, so that one multicast commit reaches them
+constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
+constexpr uint32_t kBarBytes = 512;
+constexpr int kSmemPlanItems = 128;
+constexpr uint32_t kOffPlan = kOffBars + kBarBytes;
+constexpr uint32_t kOffSeqlens = kOffPlan + ((kSmemPlanItems + 1) * 4 + 15) / 16 * 16;
+constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
+static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
+static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0 && kOffStage % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kQCol = 0;            // score CTA: latent part of Q, 256 columns (two bf16 per column)
+constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 columns
+
+constexpr uint16_t kMaskScore = 0x3, kMaskValue = 0xC, kMaskAll = 0xF;
+
+// X_PV exists in all four CTAs: PVDONE in the value CTAs, "P buffer free" in the score CTAs.  Barriers marked (L)
+// are used in the pair's even CTA only; the odd CTA's warps arrive on them remotely.
+enum { X_PV = 0, X_COMMON = X_PV + kNumP };
+enum { A_KFULL = X_COMMON /*L*/, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2 /*L*/,
+       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2 /*L*/, A_QFREE, A_NUM };
+enum { B_VFULL = X_COMMON /*L*/, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP /*L*/,
+       B_NUM = B_OREADY + kNumP };
+static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
+
+struct Unit {
+  int b, r0, n_b, t0, t1, slot;    // r0: first row of the 256-row block; t0, t1: 128-key tiles
+};
+
+struct UnitIter {
+  const DecodeParams& prm;
+  Plan plan;
+  int p, g, g1;
+  const int* seqlens;
+  __device__ UnitIter(const DecodeParams& prm_, const int* prefix, const int* seqlens_, int part)
+      : prm(prm_), plan(Plan::make(prefix, prm_.n_items, prm_.P, prm_.ovh)), p(part), seqlens(seqlens_) {
+    if (plan.L <= 0 || p >= plan.P) { g = g1 = 0; }
+    else { g = plan.part_start(p); g1 = plan.part_start(p + 1); }
+  }
+  __device__ bool next(Unit& u) {
+    int it, a;
+    while (true) {
+      if (g >= g1) return false;
+      it = plan.item_of_tile(g);
+      a = plan.first_tile(it);
+      const int e = plan.prefix[it + 1];
+      const int lo = max(g, a), hi = min(e, g1);
+      g = min(e, g1);
+      if (hi > lo) { u.t0 = lo - a; u.t1 = hi - a; break; }
+    }
+    u.b = it / prm.nrb;
+    u.r0 = (it % prm.nrb) * kItemRows;
+    u.n_b = min(max(seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
+    int p_first, p_last;
+    const int nsplit = plan.item_parts(it, &p_first, &p_last);
+    u.slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
+    return true;
+  }
+};
+
+// Finds the unit that holds the k-th tile of this cluster's part; k never decreases between calls.
+struct Cursor {
+  UnitIter it;
+  Unit u;
+  int base;
+  bool valid;
+  __device__ Cursor(const DecodeParams& prm, const int* prefix, const int* seqlens, int part) : it(prm, prefix, seqlens, part), base(0) { valid = it.next(u); }
+  __device__ bool locate(int k, int& local) {
+    while (valid && k >= base + (u.t1 - u.t0)) { base += u.t1 - u.t0; valid = it.next(u); }
+    local = k - base;
+    return valid;
+  }
+};
+
+__device__ __forceinline__ void report_timeout(int* status) { atomicExch(status, kStatusTimeout); }
+
+template <bool kClusterAcquire = false>
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, mbar_wait<kClusterAcquire>(bar, parity));
+}
+
+// One arrival per warp on a barrier of the pair's even CTA, after every lane's preceding work.
+__device__ __forceinline__ void warp_arrive_cluster(uint32_t cluster_bar, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive_cluster(cluster_bar);
+}
+
+__device__ __forceinline__ void prefetch_q_row(const DecodeParams& prm, const Unit& u, int row) {
+  if (u.r0 + row < prm.R) {
+    const char* p = reinterpret_cast<const char*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + row) * kDqk);
+#pragma unroll
+    for (int i = 0; i < 9; ++i) prefetch_l2(p + 128 * i);
+  }
+}
+
+// One query row: four 64-column blocks [blk0, blk0 + 4) of its latent part, global memory -> tensor memory.
+__device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int blk0, uint32_t taddr) {
+#pragma unroll 1
+  for (int b = blk0; b < blk0 + 4; b += 2) {
+    uint32_t x0[32], x1[32];
+    if (valid) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        ldg_256(qrow + b * 8 + 2 * c, x0, 8 * c);
+        ldg_256(qrow + b * 8 + 8 + 2 * c, x1, 8 * c);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) { x0[i] = 0; x1[i] = 0; }
+    }
+    tmem_st_32x32b_x32(taddr + b * 32, x0);
+    tmem_st_32x32b_x32(taddr + b * 32 + 32, x1);
+  }
+}
+
+struct RoleCtx {
+  uint32_t smem_base, bars, tbase, lead_bars;   // lead_bars: barrier area of the pair's even CTA (cluster address)
+  int half, tid;                                // half: which 128 rows of the 256-row block this CTA owns
+};
+
+// The softmax warpgroup's work on one unit: its 128-key score tiles; the final scalars travel with the last page.
+// Returns (pages so far) << 32 | (score tiles so far) << 1 | ok.
+template <int kMode>
+__device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const RoleCtx c, const Unit u, uint32_t gt, uint32_t gs) {
+  const int tid = c.tid, wid = tid >> 5, lane = tid & 31;
+  const uint32_t smem_base = c.smem_base, bars = c.bars, tbase = c.tbase;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  bool ok = true;
+  const int r = tid;
+  const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+  const bool scale_nonneg = prm.scale_log2 >= 0.f;
+  const uint32_t mask_fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
+  RowState st;
+  row_state_init(st);
+  const int tok = (u.r0 + c.half * kRowBlock + r) / prm.H;
+  const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);               // keys 0..visible-1 are seen by this row
+  const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kTileKeys;   // tiles from here on may hold hidden keys
+
+  for (int t = u.t0; t < u.t1 && ok; ++t, ++gs) {
+    const uint32_t sb = gs & 1;
+    ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
+    if (!ok) break;
+    tc_fence_after_sync();
+    const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
+    const int nvis = visible - t * kTileKeys;            // keys of this tile the row sees (may be <= 0)
+    const bool last_tile = t + 1 == u.t1;
+    auto tile_body = [&](auto general_c) {
+      constexpr bool kGeneral = decltype(general_c)::value;
+      constexpr bool masked = kGeneral;
+      const bool scale_nn = kGeneral ? scale_nonneg : true;
+      uint32_t b0[32], b1[32];
+      // lines 5-6: running max on the raw scores (the scale is folded into the FMA below)
+      float ext = scale_nn ? -INFINITY : INFINITY, ext_b = ext;
+      auto chunk_max = [&](uint32_t (&v)[32], int col0) {
+        if (masked) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = (col0 + i < nvis) ? v[i] : mask_fill;
+        }
+        if (scale_nn) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            ext = fmax3(ext, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            ext_b = fmax3(ext_b, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            ext = fminf(ext, fminf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+            ext_b = fminf(ext_b, fminf(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3])));
+          }
+        }
+      };
+      tmem_ld_32x32b_x32(scol, b0);
+#pragma unroll 1
+      for (int h = 0; h < 2; ++h) {
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+        chunk_max(b0, 64 * h);
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + (h == 0 ? 64 : 0), b0);   // second page, or the first chunk again for the second pass
+        chunk_max(b1, 64 * h + 32);
+      }
+      ext = scale_nn ? fmaxf(ext, ext_b) : fminf(ext, ext_b);
+      const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
+      const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
+      // Line 10's factor S16 goes into the exponential's argument (the remark after Algorithm 2).  The row sum of
+      // line 6 is the sum of the same FP32 values, taken before the bf16 cast and divided by S16 once per tile.
+      const float nsub = log2f_approx(sp.p_scale) - sp.m2_sub;
+      float rs0 = 0.f, rs1 = 0.f;
+      const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
+      uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
+      uint32_t pk[32];
+      auto chunk_exp = [&](const uint32_t (&v)[32], int col0, int k0) {
+        if (masked) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), prm.scale_log2, nsub));
+            float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), prm.scale_log2, nsub));
+            p0 = (col0 + 2 * i < nvis) ? p0 : 0.f;
+            p1 = (col0 + 2 * i + 1 < nvis) ? p1 : 0.f;
+            rs0 += p0; rs1 += p1;
+            pk[k0 + i] = pack_bf16x2(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float x0, x1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sc2, ns2), x0, x1);
+            const float q0 = ex2_approx(x0), q1 = ex2_approx(x1);
+            const uint64_t pp = pack_f32x2(q0, q1);
+            if (i & 1) rsb = add_f32x2(rsb, pp); else rsa = add_f32x2(rsa, pp);
+            pk[k0 + i] = pack_bf16x2(q0, q1);
+          }
+        }
+      };
+#pragma unroll 1
+      for (int h = 0; h < 2; ++h) {
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+        chunk_exp(b0, 64 * h, 0);
+        tmem_wait_ld();
+        if (h == 0) {
+          tmem_ld_32x32b_x32(scol + 64, b0);
+        } else {                       // the score tile has been read for the last time
+          tc_fence_before_sync();
+          warp_arrive_cluster(c.lead_bars + 8u * (A_SEMPTY + sb), lane);
+        }
+        // One staging buffer: the copy warps of the previous page must have read it into registers.  The barrier
+        // is probed ahead of the last chunk's arithmetic, so that the probe's latency is not exposed.
+        const bool stage_free = gt == 0 || mbar_probe(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+        chunk_exp(b1, 64 * h + 32, 16);
+        const uint32_t s2 = gt & 1;
+        if (!__all_sync(0xffffffffu, stage_free)) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+        if (!ok) break;
+        const uint32_t stg = smem_base + kOffStage;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc)
+          st_shared_v4(stg + sw128_offset(r, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+        // the rescale (if any) belongs to the first page; the second leaves O alone
+        const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
+                                            : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
+        st_shared_b32(stg + kNOff + r * 4, nword);
+        if (h == 1) {
+          float s0, s1;
+          unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
+          st.l = st.l * sp.l_up + __fdividef((rs0 + s0) + (rs1 + s1), sp.p_scale);
+          if (last_tile) {
+            // line 20 scalars: 1 / (l * S16) and lse = m + ln l; they ride with the unit's last page
+            const bool live = st.l > 0.f;
+            const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
+            const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(stg + kFinOff + r * 8), "r"(__float_as_uint(inv)), "r"(__float_as_uint(lse)) : "memory");
+          }
+        }
+        mbar_arrive(bar(A_PSTAGED + s2));
+        ++gt;
+      }
+    };
+    if (t >= first_masked_tile || !scale_nonneg) tile_body(std::true_type{});
+    else tile_body(std::false_type{});
+  }
+  return (static_cast<uint64_t>(gt) << 32) | (static_cast<uint64_t>(gs) << 1) | (ok ? 1u : 0u);
+}
+
+}  // namespace
+
+template <int kMode, bool kGuard>
+__global__ void __cluster_dims__(4, 1, 1) __launch_bounds__(kThreads, 1)
+decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const DecodeParams prm) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = smem_u32(smem_raw);
+  const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool is_score = rank < 2;
+  const int half = rank & 1;                 // which 128 rows of the block; the even CTA of a pair issues its MMAs
+  const bool leader = half == 0;
+  const int part = blockIdx.x >> 2;
+  if (smem_base & 1023u) {
+    if (tid == 0) report_timeout(prm.status);
+    return;
+  }
+
+  const uint32_t bars = smem_base + kOffBars;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  const uint32_t tmem_slot = bars + kBarBytes - 8;
+  const uint32_t lead_bars = map_to_cta(bars, rank & ~1u);              // barrier area of this pair's even CTA
+  const uint32_t myV_base = map_to_cta(smem_base, 2 + half);           // score CTA j -> value CTA j
+  const uint32_t myV_bars = map_to_cta(bars, 2 + half);
+
+  if (tid == 0) {
+    for (int i = 0; i < kNumP; ++i) mbar_init(bar(X_PV + i), 1);
+    if (is_score) {
+      for (int i = 0; i < kNumKSlots; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 8);         // 4 softmax warps of either CTA
+        mbar_init(bar(A_PSTAGED + i), 128); mbar_init(bar(A_STAGEFREE + i), 2);
+      }
+      mbar_init(bar(A_QREADY), 16);                                              // 8 loading warps of either CTA
+      mbar_init(bar(A_QFREE), 1);
+    } else {
+      for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
+      for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 16); }   // 8 correction warps of either CTA
+    }
+    fence_mbar_init();
+    prefetch_tensormap(&k_map);
+    prefetch_tensormap(&v_map);
+  }
+  if (wid == 5) { tmem_alloc_pair(tmem_slot, kTmemCols); tmem_relinquish_pair(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after_sync();
+  const uint32_t tbase = ld_shared_b32(tmem_slot);
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;");
+  const int* prefix = prm.prefix;
+  const int* seqlens = prm.seqlens;
+  if (prm.fused_plan) {
+    int* ps = prm.n_items <= kSmemPlanItems ? reinterpret_cast<int*>(smem_raw + kOffPlan) : nullptr;
+    if (wid == 6) {
+      int* pw = const_cast<int*>(prm.prefix);
+      int carry = 0;
+      for (int base = 0; base < prm.n_items; base += 32) {
+        const int it = base + lane;
+        const int n_seq = it < prm.n_items ? prm.seqlens[it / prm.nrb] : 0;
+        if (ps && it < prm.n_items) reinterpret_cast<int*>(smem_raw + kOffSeqlens)[it / prm.nrb] = n_seq;
+        const int v = it < prm.n_items ? schedule_length(n_seq, it, prm.tile_keys, prm.ovh) : 0;
+        int x = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, x, o);
+          if (lane >= o) x += y;
+        }
+        if (it < prm.n_items) {
+          pw[it] = carry + x - v;
+          if (ps) ps[it] = carry + x - v;
+        }
+        carry += __shfl_sync(0xffffffffu, x, 31);
+      }
+      if (lane == 0) {
+        pw[prm.n_items] = carry;
+        if (ps) ps[prm.n_items] = carry;
+        if (blockIdx.x == 0) *prm.status = kStatusOk;
+      }
+      __threadfence_block();
+    }
+    __syncthreads();
+    if (ps) { prefix = ps; seqlens = reinterpret_cast<const int*>(smem_raw + kOffSeqlens); }
+  }
+  if (is_score && tid < kRowBlock) {
+    UnitIter first(prm, prefix, seqlens, part);
+    Unit fu;
+    if (first.next(fu)) prefetch_q_row(prm, fu, half * kRowBlock + tid);
+  }
+
+  bool ok = true;
+  UnitIter iter(prm, prefix, seqlens, part);
+  Unit u;
+  uint32_t gt = 0;      // 64-key pages processed by this cluster so far (two per tile; all roles count identically)
+  uint32_t un = 0;      // units processed so far
+
+  if (is_score) {
+    // ======================================================================= score CTAs
+    uint32_t gs = 0;    // score tiles so far
+    if (wid < 4) {
+      // ---- softmax warpgroup: thread = query row
+      const int r = tid;
+      const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+      const RoleCtx ctx{smem_base, bars, tbase, lead_bars, half, tid};
+      while (ok && iter.next(u)) {
+        ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);      // the previous unit's QK^T is finished with Q
+        if (!ok) break;
+        tc_fence_after_sync();
+        {
+          const int row = u.r0 + half * kRowBlock + r;
+          const bool valid = row < prm.R;
+          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDqk);
+          load_q_latent(qrow, valid, 0, tbase + lane_base + kQCol);
+          tmem_wait_st();
+        }
+        tc_fence_before_sync();
+        warp_arrive_cluster(lead_bars + 8u * A_QREADY, lane);
+        const uint64_t ret = softmax_unit<kMode>(prm, ctx, u, gt, gs);
+        gt = static_cast<uint32_t>(ret >> 32);
+        gs = static_cast<uint32_t>(ret & 0xffffffffu) >> 1;
+        ok = (ret & 1u) != 0;
+        ++un;
+      }
+      if (!ok) report_timeout(prm.status);
+    } else if (wid == 4) {
+      // ---- TMA producers: K.  This CTA loads page (2 t + half) of every tile t, three slots of 192 columns; lane l
+      // owns ring slot l and polls without blocking.  The bytes of both CTAs' halves are counted on the even CTA's
+      // "full" barrier.  A sequence's last tile may have one page only: the odd CTA then loads the first page
+      // again (finite values that the softmax masks as keys beyond the sequence).
+      Cursor cur(prm, prefix, seqlens, part);
+      int my_tile = lane / 3;                 // kNumKSlots = 6: lane l always loads column group l % 3, every second tile
+      const int g = lane % 3;
+      uint32_t par = 1;
+      bool fin = lane >= kNumKSlots, have = false;
+      int page_id = 0;
+      int issued = 0;
+      const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane);
+      const uint32_t lead_full = lead_bars + 8u * (A_KFULL + lane);
+      const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
+      uint64_t t_start = global_timer_ns();
+      bool progress = false;
+      for (uint32_t spin = 0;; ++spin) {
+        if (!fin && !have) {
+          int lt;
+          if (cur.locate(my_tile, lt)) {
+            const int t = cur.u.t0 + lt;
+            const int npg = (cur.u.n_b + kPage - 1) / kPage;
+            const int pg = (2 * t + half < npg) ? 2 * t + half : 2 * t;
+            page_id = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + pg);
+            have = true;
+          } else {
+            fin = true;
+          }
+        }
+        if (have && mbar_probe(my_empty, par)) {
+          if (leader) mbar_arrive_expect_tx(my_full, 2 * kKSlotBytes);
+          tma_load_4d_pair(dst, &k_map, 0, 0, 3 * g, page_id * 8, lead_full);
+          my_tile += 2;
+          par ^= 1;
+          ++issued;
+          have = false;
+          progress = true;
+        }
+        if (__all_sync(0xffffffffu, fin)) break;
+        const bool any_progress = __any_sync(0xffffffffu, progress);
+        if (any_progress) t_start = global_timer_ns(); else __nanosleep(100);
+        progress = false;
+        if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) { ok = false; break; }
+      }
+      if (!ok) {
+        if (lane == 0) report_timeout(prm.status);
+        if (leader && issued > 0 && lane < kNumKSlots) mbar_wait(my_full, (issued - 1) & 1);   // let copies in flight land
+      }
+    } else if (wid == 5) {
+      // ---- MMA issuer (even CTA only): S[sb] = Q K^T for both CTAs' rows, 36 steps of K = 16 over three slots
+      if (leader && lane == 0) {
+        constexpr uint32_t idesc = make_idesc_bf16(256, 128, false, false);
+        constexpr uint32_t dhi = smem_desc_hi_sw128(kKGroupStride);
+        constexpr uint32_t qhi = smem_desc_hi_sw128(1024);
+        const uint32_t klo0 = smem_desc_lo(smem_base + kOffK, 16);
+        const uint32_t qlo0 = smem_desc_lo(smem_base + kOffQRope, 16);
+        uint32_t slot = 0, kpar = 0;
+        while (ok && iter.next(u)) {
+          ok = mbar_wait<true>(bar(A_QREADY), un & 1);
+          if (!ok) break;
+          tc_fence_after_sync();
+          for (int t = u.t0; t < u.t1 && ok; ++t, ++gs) {
+            const uint32_t sb = gs & 1;
+            ok = mbar_wait<true>(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t d = tbase + kSCol + 128 * sb;
+#pragma unroll
+            for (int gg = 0; gg < 3; ++gg) {
+              ok = ok && mbar_wait<true>(bar(A_KFULL) + 8 * slot, kpar);
+              if (ok) {
+                const uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
+#pragma unroll
+                for (int cl = 0; cl < 3; ++cl) {
+                  const int cb = 3 * gg + cl;
+#pragma unroll
+                  for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t bd = smem_desc_join(klo + 64 * cl + 2 * kk, dhi);
+                    if (cb < 8) mma_ts_pair(d, tbase + kQCol + 32 * cb + 8 * kk, bd, idesc, (cb | kk) != 0 ? 1u : 0u);
+                    else mma_ss_pair(d, smem_desc_join(qlo0 + 2 * kk, qhi), bd, idesc, 1u);   // RoPE columns: Q from shared memory
+                  }
+                }
+                mma_commit_pair_multicast(bar(A_KEMPTY) + 8 * slot, kMaskScore);
+              }
+              if (++slot == kNumKSlots) { slot = 0; kpar ^= 1; }
+            }
+            if (!ok) break;
+            mma_commit_pair_multicast(bar(A_SFULL + sb), kMaskScore);
+          }
+          if (!ok) break;
+          mma_commit_pair_multicast(bar(A_QFREE), kMaskScore);
+          ++un;
+        }
+        if (!ok) report_timeout(prm.status);
+      }
+    } else if (wid >= 6 && wid < 6 + kNumCopyWarps) {
+      // ---- copy warps: staged P~ / N (and, with a unit's last page, the final scalars) -> a free P buffer of this
+      // CTA's value CTA, by asynchronous remote stores counted on its PFULL barrier.  Warps c and c + 2 serve the
+      // pages of parity c and move one half of the buffer each.
+      const uint32_t c = (wid - 6) & 1, hv = (wid - 6) >> 1;
+      constexpr int kChunks = 18;                         // 512-byte chunks per warp (33 or 35 in total)
+      const int qr = (wid & 3) * 32 + lane;
+      const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+      while (ok && iter.next(u)) {
+        {
+          ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const int row = u.r0 + half * kRowBlock + qr;
+          const bool valid = row < prm.R;
+          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDqk);
+          load_q_latent(qrow, valid, 4, tbase + q_lane_base + kQCol);
+#pragma unroll
+          for (int cc = 0; cc < 8; ++cc) {
+            const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
+            st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
+          }
+          tmem_wait_st();
+          fence_proxy_async_smem();
+          tc_fence_before_sync();
+          warp_arrive_cluster(lead_bars + 8u * A_QREADY, lane);
+          ++un;
+          UnitIter peek = iter;
+          Unit nu;
+          if (peek.next(nu)) prefetch_q_row(prm, nu, half * kRowBlock + qr);
+        }
+        const int npages = 2 * (u.t1 - u.t0);
+        for (int pi = 0; pi < npages; ++pi, ++gt) {
+          if ((gt & 1) != c) continue;
+          const bool last = pi + 1 == npages;
+          const int nchunks = last ? 35 : 33;
+          const uint32_t pb = gt % kNumP;
+          ok = warp_wait(bar(A_PSTAGED + c), (gt >> 1) & 1);
+          if (!ok) break;
+          const uint32_t src = smem_base + kOffStage + (hv * kChunks * 32 + lane) * 16;
+          uint32_t v[kChunks][4];
+#pragma unroll
+          for (int i = 0; i < kChunks; ++i) {
+            if (static_cast<int>(hv) * kChunks + i < nchunks)
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i][0]), "=r"(v[i][1]), "=r"(v[i][2]), "=r"(v[i][3]) : "r"(src + i * 512));
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(A_STAGEFREE + c));
+          ok = warp_wait(bar(X_PV + pb), ((gt / kNumP) & 1) ^ 1);      // the P V that last read the buffer is done
+          if (!ok) break;
+          const uint32_t pfull = myV_bars + 8u * (B_PFULL + pb);
+          const uint32_t dstp = myV_base + kOffP + pb * kPStride + (hv * kChunks * 32 + lane) * 16;
+          if (lane == 0 && hv == 0) mbar_arrive_expect_tx_cluster(pfull, last ? kPXferLast : kPXfer);
+#pragma unroll
+          for (int i = 0; i < kChunks; ++i) {
+            if (static_cast<int>(hv) * kChunks + i < nchunks) st_async_v4(dstp + i * 512, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
+          }
+        }
+      }
+      if (!ok && lane == 0) report_timeout(prm.status);
+    }
+  } else {
+    // ======================================================================= value CTAs
+    if (wid < 4 || (wid >= 6 && wid < 10)) {
+      // ---- correction + epilogue: thread = query row.  Warps 6-9 are the partners of warps 2, 3, 0, 1 (same
+      // tensor-memory lanes): each of a pair rescales one half of the row's 512 columns.  Epilogue: warps 0-3.
+      const bool partner = wid >= 4;
+      const int r = (wid & 3) * 32 + lane;
+      const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+      const int c_first = partner ? 8 : 0;
+      while (ok && iter.next(u)) {
+        const int npages = 2 * (u.t1 - u.t0);
+        float inv = 0.f, lse = 0.f;
+        for (int pi = 0; pi < npages && ok; ++pi, ++gt) {
+          const uint32_t s = gt % kNumP, k = gt / kNumP;
+          ok = warp_wait<true>(bar(B_PFULL + s), k & 1);
+          if (!ok) break;
+          const uint32_t pbuf = smem_base + kOffP + s * kPStride;
+          const uint32_t nword = ld_shared_b32(pbuf + kNOff + r * 4);
+          if (pi + 1 == npages && !partner) {
+            uint32_t x, y;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(pbuf + kFinOff + r * 8));
+            inv = __uint_as_float(x); lse = __uint_as_float(y);
+          }
+          const bool mine = (kMode == 2) ? (__uint_as_float(nword) != 1.f) : (nword != 0u);
+          if (__any_sync(0xffffffffu, mine) && pi > 0) {
+            // lines 13-16: O <- AS_FP32(AS_INT32(O) + N), after P V of the previous page has landed
+            const uint32_t gp = gt - 1;
+            ok = warp_wait(bar(X_PV + gp % kNumP), (gp / kNumP) & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            auto apply = [&](uint32_t (&o)[32]) {
+              if (kMode == 2) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * __uint_as_float(nword));
+              } else if (!kGuard) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(exponent_add_raw(__uint_as_float(o[i]), static_cast<int>(nword)));
+              } else {
+                // the guard matters only where magnitude bits + N would not stay positive: take the chunk's smallest
+                // magnitude first and use the plain one-instruction add of Lemma 3.1 where it is safe
+                float lo = fmin3_abs(__uint_as_float(o[0]), __uint_as_float(o[1]), __uint_as_float(o[2]));
+#pragma unroll
+                for (int i = 3; i + 1 < 32; i += 2) lo = fmin3_abs(lo, __uint_as_float(o[i]), __uint_as_float(o[i + 1]));
+                lo = fminf(lo, fabsf(__uint_as_float(o[31])));
+                if (__float_as_int(lo) + static_cast<int>(nword) > 0) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(exponent_add_raw(__uint_as_float(o[i]), static_cast<int>(nword)));
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(exponent_add_guarded(__uint_as_float(o[i]), static_cast<int>(nword)));
+                }
+              }
+            };
+            uint32_t o0[32], o1[32];
+            const uint32_t obase = tbase + lane_base + 32 * c_first;
+            tmem_ld_32x32b_x32(obase, o0);
+#pragma unroll 1
+            for (int cc = 0; cc < 8; cc += 2) {
+              tmem_wait_ld();
+              tmem_ld_32x32b_x32(obase + 32 * (cc + 1), o1);
+              apply(o0);
+              tmem_st_32x32b_x32(obase + 32 * cc, o0);
+              tmem_wait_ld();
+              if (cc + 2 < 8) tmem_ld_32x32b_x32(obase + 32 * (cc + 2), o0);
+              apply(o1);
+              tmem_st_32x32b_x32(obase + 32 * (cc + 1), o1);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+          }
+          // this CTA's P~ (remote asynchronous stores, generic proxy) is about to be read by the pair MMA
+          fence_proxy_async_smem();
+          warp_arrive_cluster(lead_bars + 8u * (B_OREADY + s), lane);
+        }
+        if (!ok) break;
+        // ---- epilogue (line 20): out = O / (l * S16)
+        if (!partner) {
+          const uint32_t gl = gt - 1;
+          ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const int row0 = u.r0 + half * kRowBlock;               // first row of this CTA within the sequence
+          const bool valid = row0 + r < prm.R;
+          const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
+          const int rows_here = min(32, prm.R - row0 - wid * 32);
+          __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + row0 + wid * 32) * kDv;
+          float* pbase = prm.part_o + (static_cast<size_t>(u.slot < 0 ? 0 : u.slot) * kItemRows + half * kRowBlock + wid * 32) * kDv;
+          uint32_t o[2][32];
+          tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
+#pragma unroll 1
+          for (int cq = 0; cq < 16; cq += 2) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              tmem_wait_ld();
+              if (cq + e + 1 < 16) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (cq + e + 1), o[e ^ 1]);
+              const int cc = cq + e;
+              __syncwarp();
+              if (u.slot < 0) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                  const uint32_t w0 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 0]) * inv, __uint_as_float(o[e][8 * jj + 1]) * inv);
+                  const uint32_t w1 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 2]) * inv, __uint_as_float(o[e][8 * jj + 3]) * inv);
+                  const uint32_t w2 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 4]) * inv, __uint_as_float(o[e][8 * jj + 5]) * inv);
+                  const uint32_t w3 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 6]) * inv, __uint_as_float(o[e][8 * jj + 7]) * inv);
+                  st_shared_v4(epi + lane * 128 + ((jj ^ (lane & 7)) << 4), w0, w1, w2, w3);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int kq = 0; kq < 4; ++kq) {                       // 8 rows x 64 B per instruction
+                  const int row = 8 * kq + (lane >> 2), jj = lane & 3;
+                  uint4 v;
+                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                               : "r"(epi + row * 128 + ((jj ^ (row & 7)) << 4)));
+                  if (row < rows_here) *reinterpret_cast<uint4*>(obase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * jj) = v;
+                }
+              } else {
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj)
+                  st_shared_v4(epi + lane * 128 + ((jj ^ (lane & 7)) << 4),
+                               __float_as_uint(__uint_as_float(o[e][4 * jj + 0]) * inv), __float_as_uint(__uint_as_float(o[e][4 * jj + 1]) * inv),
+                               __float_as_uint(__uint_as_float(o[e][4 * jj + 2]) * inv), __float_as_uint(__uint_as_float(o[e][4 * jj + 3]) * inv));
+                __syncwarp();
+#pragma unroll
+                for (int kq = 0; kq < 8; ++kq) {                       // 4 rows x 128 B per instruction
+                  const int row = 4 * kq + (lane >> 3), jj = lane & 7;
+                  uint4 v;
+                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                               : "r"(epi + row * 128 + ((jj ^ (row & 7)) << 4)));
+                  if (row < rows_here) *reinterpret_cast<uint4*>(pbase + static_cast<size_t>(row) * kDv + 32 * cc + 4 * jj) = v;
+                }
+              }
+            }
+          }
+          if (valid) {
+            if (u.slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + row0 + r] = lse;
+            else prm.part_lse[static_cast<size_t>(u.slot) * kItemRows + half * kRowBlock + r] = lse;
+          }
+          tc_fence_before_sync();
+        }
+        ++un;
+      }
+      if (!ok) report_timeout(prm.status);
+    } else if (wid == 4) {
+      // ---- TMA producers: V.  One slot per page: this CTA's 128 columns of either 256-column half of V (two
+      // boxes of 64 keys x 128 columns); lane l owns ring slot l.  Both pages of every tile are loaded (the
+      // second page of a sequence's odd last tile is the first one again; its probabilities are zero).
+      Cursor cur(prm, prefix, seqlens, part);
+      int my_gp = lane;                       // next page of the sequence this lane loads (tile = gp / 2)
+      uint32_t par = 1;
+      bool fin = lane >= kNumVSlots, have = false;
+      int page_id = 0;
+      int issued = 0;
+      const uint32_t my_full = bar(B_VFULL + lane), my_empty = bar(B_VEMPTY + lane);
+      const uint32_t lead_full = lead_bars + 8u * (B_VFULL + lane);
+      const uint32_t dst = smem_base + kOffV + lane * kVSlotBytes;
+      uint64_t t_start = global_timer_ns();
+      bool progress = false;
+      for (uint32_t spin = 0;; ++spin) {
+        if (!fin && !have) {
+          int lt;
+          if (cur.locate(my_gp >> 1, lt)) {
+            const int t = cur.u.t0 + lt;
+            const int npg = (cur.u.n_b + kPage - 1) / kPage;
+            const int pg = (2 * t + (my_gp & 1) < npg) ? 2 * t + (my_gp & 1) : 2 * t;
+            page_id = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + pg);
+            have = true;
+          } else {
+            fin = true;
+          }
+        }
+        if (have && mbar_probe(my_empty, par)) {
+          if (leader) mbar_arrive_expect_tx(my_full, 2 * kVSlotBytes);
+          tma_load_3d_pair(dst, &v_map, 0, page_id * kPage, 2 * half, lead_full);
+          tma_load_3d_pair(dst + kVHalfBytes, &v_map, 0, page_id * kPage, 4 + 2 * half, lead_full);
+          my_gp += kNumVSlots;
+          par ^= 1;
+          ++issued;
+          have = false;
+          progress = true;
+        }
+        if (__all_sync(0xffffffffu, fin)) break;
+        const bool any_progress = __any_sync(0xffffffffu, progress);
+        if (any_progress) t_start = global_timer_ns(); else __nanosleep(100);
+        progress = false;
+        if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) { ok = false; break; }
+      }
+      if (!ok) {
+        if (lane == 0) report_timeout(prm.status);
+        if (leader && issued > 0 && lane < kNumVSlots) mbar_wait(my_full, (issued - 1) & 1);
+      }
+    } else if (wid == 5) {
+      // ---- MMA issuer (even CTA only): O (+)= P~ V for both CTAs' rows; per page two N = 256 halves of four
+      // K = 16 steps
+      if (leader && lane == 0) {
+        constexpr uint32_t idesc = make_idesc_bf16(256, 256, false, true);
+        constexpr uint32_t dhi = smem_desc_hi_sw128(1024);
+        const uint32_t vlo0 = smem_desc_lo(smem_base + kOffV, kBoxBytes);
+        const uint32_t plo0 = smem_desc_lo(smem_base + kOffP, 16);
+        uint32_t slot = 0, vpar = 0;
+        while (ok && iter.next(u)) {
+          const int npages = 2 * (u.t1 - u.t0);
+          for (int pi = 0; pi < npages && ok; ++pi, ++gt) {
+            const uint32_t s = gt % kNumP, k = gt / kNumP;
+            ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
+            if (!ok) break;
+            ok = mbar_wait<true>(bar(B_OREADY + s), k & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            fence_proxy_async_smem();
+            ok = mbar_wait<true>(bar(B_VFULL) + 8 * slot, vpar);
+            if (!ok) break;
+            const uint32_t plo = plo0 + s * (kPStride >> 4);
+            const uint32_t vlo = vlo0 + slot * (kVSlotBytes >> 4);
+            const uint32_t acc0 = pi > 0 ? 1u : 0u;
+#pragma unroll
+            for (int nh = 0; nh < 2; ++nh) {
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                mma_ss_pair(tbase + nh * 256, smem_desc_join(plo + 2 * kk, dhi), smem_desc_join(vlo + nh * (kVHalfBytes >> 4) + 128 * kk, dhi),
+                            idesc, kk == 0 ? acc0 : 1u);
+            }
+            mma_commit_pair_multicast(bar(B_VEMPTY) + 8 * slot, kMaskValue);
+            if (++slot == kNumVSlots) { slot = 0; vpar ^= 1; }
+            mma_commit_pair_multicast(bar(X_PV + s), kMaskAll);   // PVDONE in the value CTAs, "P buffer free" in the score CTAs
+          }
+          if (!ok) break;
+        }
+        if (!ok) report_timeout(prm.status);
+      }
+    }
+  }
+
+  // teardown: nobody may still be writing into a CTA that has exited, and both CTAs of a pair must be done
+  // with tensor memory before it is freed
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (wid == 5) tmem_dealloc_pair(tbase, kTmemCols);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static std::atomic<EncodeTiledFn> fn{nullptr};
+  EncodeTiledFn f = fn.load(std::memory_order_acquire);
+  if (!f) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess) {
+      f = reinterpret_cast<EncodeTiledFn>(p);
+      fn.store(f, std::memory_order_release);
+    }
+  }
+  return f;
+}
+
+void fill_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int clusters, cudaStream_t stream) {
+  cfg = cudaLaunchConfig_t{};
+  cfg.gridDim = dim3(4 * clusters);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+}
+
+template <int kMode, bool kGuard>
+cudaError_t prepare_variant(int device) {
+  static std::atomic<uint64_t> done{0};
+  const uint64_t bit = 1ull << (device & 63);
+  if (!(done.load(std::memory_order_acquire) & bit)) {
+    const cudaError_t err = cudaFuncSetAttribute(decode_quad_kernel<kMode, kGuard>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+    if (err != cudaSuccess) return err;
+    done.fetch_or(bit, std::memory_order_release);
+  }
+  return cudaSuccess;
+}
+
+template <int kMode, bool kGuard>
+cudaError_t launch_variant(const CUtensorMap& kmap, const CUtensorMap& vmap, const DecodeParams& prm, cudaStream_t stream) {
+  int device = 0;
+  cudaError_t err = cudaGetDevice(&device);
+  if (err != cudaSuccess) return err;
+  err = prepare_variant<kMode, kGuard>(device);
+  if (err != cudaSuccess) return err;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fill_config(cfg, attr, prm.P, stream);
+  return cudaLaunchKernelEx(&cfg, decode_quad_kernel<kMode, kGuard>, kmap, vmap, prm);
+}
+
+}  // namespace
+
+// Number of four-CTA clusters that can be resident at once on `device` (0 if the query fails): the parts the
+// schedule is cut into.  Queried once per device.
+int decode_quad_parts(int device, int sm_count) {
+  static std::atomic<int> cache[64];
+  if (device < 0 || device >= 64) return 0;
+  int v = cache[device].load(std::memory_order_acquire);
+  if (v > 0) return v;
+  if (prepare_variant<0, true>(device) != cudaSuccess) { cudaGetLastError(); return 0; }
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fill_config(cfg, attr, sm_count / 4 > 0 ? sm_count / 4 : 1, nullptr);
+  cfg.numAttrs = 0;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, decode_quad_kernel<0, true>, &cfg) != cudaSuccess || n <= 0) { cudaGetLastError(); return 0; }
+  if (n > sm_count / 4) n = sm_count / 4;
+  cache[device].store(n, std::memory_order_release);
+  return n;
+}
+
+cudaError_t launch_decode_quad(const DecodeParams& prm, cudaStream_t stream, int* unsupported) {
+  *unsupported = 0;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) { *unsupported = 1; return cudaErrorNotSupported; }
+  // K: the cache seen as (64 columns, 8 rows of a group, 9 column blocks, row groups); one box = a page's 64 keys x
+  // 3 column blocks, laid out in shared memory as [row group][column block][8 keys][64 columns], so that a
+  // K-major operand descriptor with a group stride of 3 KB walks the keys of one column block.
+  CUtensorMap kmap;
+  {
+    const cuuint64_t dims[4] = {64, 8, static_cast<cuuint64_t>(kDqk / 64), static_cast<cuuint64_t>(prm.num_blocks) * 8};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kDqk) * 2, 128, static_cast<cuuint64_t>(kDqk) * 2 * 8};
+    const cuuint32_t box[4] = {64, 8, 3, 8};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult cr = encode(&kmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<__nv_bfloat16*>(prm.kv), dims, strides,
+                               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+  // V: the same rows seen as (64 columns, rows, column block); one box = 64 keys x 2 column blocks, laid out in
+  // shared memory as [column block][key][64 columns]: the MN-major B operand of 128 output columns.
+  CUtensorMap vmap;
+  {
+    const cuuint64_t vdims[3] = {64, static_cast<cuuint64_t>(prm.num_blocks) * kPage, static_cast<cuuint64_t>(kDqk / 64)};
+    const cuuint64_t vstrides[2] = {static_cast<cuuint64_t>(kDqk) * 2, 128};
+    const cuuint32_t vbox[3] = {64, 64, 2};
+    const cuuint32_t vestr[3] = {1, 1, 1};
+    const CUresult vr = encode(&vmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(prm.kv), vdims, vstrides,
+                               vbox, vestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (vr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+  const int mode = prm.flags & 3;
+  const bool guard = !(prm.flags & 4);
+  if (mode == 0) return guard ? launch_variant<0, true>(kmap, vmap, prm, stream) : launch_variant<0, false>(kmap, vmap, prm, stream);
+  if (mode == 1) return guard ? launch_variant<1, true>(kmap, vmap, prm, stream) : launch_variant<1, false>(kmap, vmap, prm, stream);
+  return launch_variant<2, true>(kmap, vmap, prm, stream);
+}
+
+}  // namespace amla

@@ -21,7 +21,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
   uint32_t* Qsm = smem + kPage * kKStrideW;               // [16][288] words
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const Plan plan = Plan::make(prm.prefix, prm.n_items, prm.P);
+  const Plan plan = Plan::make(prm.prefix, prm.n_items, prm.P, prm.ovh);
   if (plan.L <= 0) return;
   const int p = blockIdx.x;
   if (p >= plan.P) return;
@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
     const int b = it / prm.nrb, rb = it % prm.nrb;
     const int r0 = rb * kRowBlock;
     const int nrows = min(kRowBlock, prm.R - r0);
-    const int n_b = prm.seqlens[b];
+    const int n_b = min(max(prm.seqlens[b], 0), prm.max_blocks_per_seq * kPage);
     int p_first, p_last;
     const int nsplit = plan.item_parts(it, &p_first, &p_last);
     const int slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);

@@ -8,10 +8,11 @@
 //       through a ring; S = Q K^T (128 x 128, FP32) by tcgen05.mma into a double-buffered TMEM tile.  The
 //       softmax warpgroup runs Algorithm 2's per-row recurrence (lines 5-12) once per score tile,
 //       writes the bf16 probabilities P~ = bf16(P * S16) of each 64-key half plus the per-row integer
-//       N into a local staging buffer, and a bulk shared-to-shared copy moves it into the value CTA.
+//       N into a local staging buffer, and four copy warps move it into the value CTA with
+//       asynchronous remote stores counted on a barrier there.
 //   value CTA (cluster rank 1)   the whole FP32 accumulator O (128 x 512) lives in its tensor memory;
 //       V (first 512 columns of the same cache rows) arrives by TMA in slots of 64 keys x 256
-//       columns through a 5-slot ring; a correction warpgroup applies N to the bit patterns of O
+//       columns through a 4-slot ring; a correction warpgroup applies N to the bit patterns of O
 //       (lines 13-16; Lemma 3.1) for rows whose reference moved, then O += P~ V by tcgen05.mma
 //       (lines 17-18); the epilogue divides by l * S16 (line 20).
 //
@@ -84,7 +85,7 @@ constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 column
 // score CTA the same arrival (multicast commit) frees the page's P buffer for the softmax (PEMPTY).
 enum { X_PV = 0, X_COMMON = X_PV + kNumP };
 enum { A_KFULL = X_COMMON, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2,
-       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2, A_QFREE, A_NUM };
+       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2, A_QFREE, A_FINFREE, A_NUM = A_FINFREE + 2 };
 enum { B_VFULL = X_COMMON, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP,
        B_FINFULL = B_OREADY + kNumP, B_NUM = B_FINFULL + 2 };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
@@ -100,7 +101,7 @@ struct UnitIter {
   int p, g, g1;
   const int* seqlens;
   __device__ UnitIter(const DecodeParams& prm_, const int* prefix, const int* seqlens_, int part)
-      : prm(prm_), plan(Plan::make(prefix, prm_.n_items, prm_.P)), p(part), seqlens(seqlens_) {
+      : prm(prm_), plan(Plan::make(prefix, prm_.n_items, prm_.P, prm_.ovh)), p(part), seqlens(seqlens_) {
     if (plan.L <= 0 || p >= plan.P) { g = g1 = 0; }
     else { g = plan.part_start(p); g1 = plan.part_start(p + 1); }
   }
@@ -347,6 +348,9 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
       else tile_body(std::false_type{});
     }
     // line 20 scalars: 1 / (l * S16) and lse = m + ln l
+    // The two-entry buffer of the value CTA is written for unit `un` only after the epilogue of unit un - 2 has read
+    // its entry (nothing else keeps this warpgroup from running two short units ahead of the epilogue).
+    if (ok) ok = warp_wait<true>(bar(A_FINFREE + (un & 1)), ((un >> 1) & 1) ^ 1);
     if (ok) {
       const bool live = st.l > 0.f;
       const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
@@ -382,6 +386,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   // addresses of the peer's barriers / buffers (same dynamic-smem base in both CTAs)
   const uint32_t peerB_bars = map_to_cta(smem_base + kOffBars, 1);
   const uint32_t peerB_base = map_to_cta(smem_base, 1);
+  const uint32_t peerA_bars = map_to_cta(smem_base + kOffBars, 0);
 
   if (tid == 0) {
     for (int i = 0; i < kNumP; ++i) mbar_init(bar(X_PV + i), 1);
@@ -393,6 +398,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       }
       mbar_init(bar(A_QREADY), 256);
       mbar_init(bar(A_QFREE), 1);
+      for (int i = 0; i < 2; ++i) mbar_init(bar(A_FINFREE + i), 4);   // the four epilogue warps of the value CTA
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
       for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 256); }
@@ -430,7 +436,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         const int it = base + lane;
         const int n_seq = it < prm.n_items ? prm.seqlens[it / prm.nrb] : 0;
         if (ps && it < prm.n_items) reinterpret_cast<int*>(smem_raw + kOffSeqlens)[it / prm.nrb] = n_seq;   // same value from every row block
-        const int v = it < prm.n_items ? schedule_length(n_seq, it) : 0;
+        const int v = it < prm.n_items ? schedule_length(n_seq, it, prm.tile_keys, prm.ovh) : 0;
         int x = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -514,7 +520,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         int issued = 0;
         const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane);
         const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
-        const uint64_t t_start = global_timer_ns();
+        uint64_t t_start = global_timer_ns();     // restarted whenever a lane issues a load: the limit bounds one stalled wait
         bool progress = false;
         for (uint32_t spin = 0;; ++spin) {
           if (!fin && !have) {
@@ -546,9 +552,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           if (__all_sync(0xffffffffu, fin)) break;
           // nothing to issue right now: back off, so that the polling does not take issue slots from the warps that
           // share this scheduler
-          if (!__any_sync(0xffffffffu, progress)) __nanosleep(100);
+          if (__any_sync(0xffffffffu, progress)) t_start = global_timer_ns(); else __nanosleep(100);
           progress = false;
-          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > 4 * kWaitLimitNs)) { ok = false; break; }
+          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) { ok = false; break; }
         }
         if (!ok) {
           if (lane == 0) report_timeout(prm.status);
@@ -789,6 +795,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(smem_base + kOffFin + ((un & 1) * 128 + r) * 8));
             inv = __uint_as_float(x); lse = __uint_as_float(y);
           }
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(peerA_bars + 8u * (A_FINFREE + (un & 1)));   // the entry may be rewritten
           const bool valid = r < u.nrows;
           // 32 columns at a time: each lane scales its row, the warp transposes the 32 x 32 tile through shared
           // memory (16-byte units XOR-swizzled by row), and writes whole 128-byte (FP32 partial) or 64-byte (bf16)
@@ -854,7 +862,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producers: V, two slots (256 columns each, one 3-D box) per page; lane l owns ring slot l
+      // ---- TMA producers: V, two ring slots per page (256 columns each, one 3-D box per slot); lane l owns ring slot l
       {
         Cursor<false> cur(prm, prefix, seqlens, part);
         int my_gv = lane;                       // next slot of the sequence this lane loads (page = gv / 2)
@@ -864,7 +872,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         int issued = 0;
         const uint32_t my_full = bar(B_VFULL + lane), my_empty = bar(B_VEMPTY + lane);
         const uint32_t dst = smem_base + kOffV + lane * kVSlotBytes;
-        const uint64_t t_start = global_timer_ns();
+        uint64_t t_start = global_timer_ns();     // restarted whenever a lane issues a load
         bool progress = false;
         for (uint32_t spin = 0;; ++spin) {
           if (!fin && !have) {
@@ -889,9 +897,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           if (__all_sync(0xffffffffu, fin)) break;
           // nothing to issue right now: back off, so that the polling does not take issue slots from the warps that
           // share this scheduler
-          if (!__any_sync(0xffffffffu, progress)) __nanosleep(100);
+          if (__any_sync(0xffffffffu, progress)) t_start = global_timer_ns(); else __nanosleep(100);
           progress = false;
-          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > 4 * kWaitLimitNs)) { ok = false; break; }
+          if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) { ok = false; break; }
         }
         if (!ok) {
           if (lane == 0) report_timeout(prm.status);

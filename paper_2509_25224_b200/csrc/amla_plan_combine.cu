@@ -9,7 +9,7 @@ namespace amla {
 // One block.  prefix[it] = sum over items before `it` of their schedule lengths (tiles plus the start-up
 // overhead of a non-empty item, see Plan); also resets the
 // status word.  n_items is small (B * ceil(Sq*H/128)); a chunked block scan covers any size.
-__global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_items,
+__global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_items, int tile_keys, int ovh,
                             int* __restrict__ prefix, int* __restrict__ status) {
   __shared__ int warp_sums[32];
   __shared__ int carry;
@@ -20,7 +20,7 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
   for (int base = 0; base < n_items; base += blockDim.x) {
     const int it = base + tid;
     int v = 0;
-    if (it < n_items) v = schedule_length(seqlens[it / nrb], it);
+    if (it < n_items) v = schedule_length(seqlens[it / nrb], it, tile_keys, ovh);
     int x = v;  // inclusive warp scan
     for (int o = 1; o < 32; o <<= 1) {
       int y = __shfl_up_sync(0xffffffffu, x, o);
@@ -54,15 +54,15 @@ __global__ void combine_kernel(DecodeParams prm) {
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row_global = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-  const int rows_padded = prm.nrb * kRowBlock;
+  const int rows_padded = prm.nrb * prm.item_rows;
   const int b = row_global / rows_padded;
   if (b >= prm.B) return;
   const int rin = row_global - b * rows_padded;   // row within the sequence, padded to row blocks
   if (rin >= prm.R) return;
-  const int rb = rin / kRowBlock, rr = rin % kRowBlock;
+  const int rb = rin / prm.item_rows, rr = rin % prm.item_rows;   // item of the sequence, row within the item
   const int it = b * prm.nrb + rb;
 
-  const Plan plan = Plan::make(prm.prefix, prm.n_items, prm.P);
+  const Plan plan = Plan::make(prm.prefix, prm.n_items, prm.P, prm.ovh);
   int p_first, p_last;
   const int nsplit = plan.L > 0 ? plan.item_parts(it, &p_first, &p_last) : 0;
   if (nsplit == 1) return;
@@ -78,7 +78,7 @@ __global__ void combine_kernel(DecodeParams prm) {
   float mx = -INFINITY;
   for (int base = 0; base < nsplit; base += 32) {
     const int sidx = base + lane;
-    if (sidx < nsplit) mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(plan.slot_of(p_first + sidx, it, p_first)) * kRowBlock + rr]);
+    if (sidx < nsplit) mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(plan.slot_of(p_first + sidx, it, p_first)) * prm.item_rows + rr]);
   }
 #pragma unroll
   for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -97,7 +97,7 @@ __global__ void combine_kernel(DecodeParams prm) {
     float my_w = 0.f;
     if (sidx < nsplit) {
       my_slot = plan.slot_of(p_first + sidx, it, p_first);
-      my_w = expf(prm.part_lse[static_cast<size_t>(my_slot) * kRowBlock + rr] - mx);   // 0 for a split that saw nothing
+      my_w = expf(prm.part_lse[static_cast<size_t>(my_slot) * prm.item_rows + rr] - mx);   // 0 for a split that saw nothing
     }
     const int n_here = min(32, nsplit - base);
 #pragma unroll 2
@@ -105,7 +105,7 @@ __global__ void combine_kernel(DecodeParams prm) {
       const float w = __shfl_sync(0xffffffffu, my_w, j);
       const int slot = __shfl_sync(0xffffffffu, my_slot, j);
       tot += w;
-      const float* src = prm.part_o + (static_cast<size_t>(slot) * kRowBlock + rr) * kDv;
+      const float* src = prm.part_o + (static_cast<size_t>(slot) * prm.item_rows + rr) * kDv;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float4 v = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
@@ -128,13 +128,13 @@ __global__ void combine_kernel(DecodeParams prm) {
 }
 
 cudaError_t launch_plan(const DecodeParams& prm, int* prefix_out, cudaStream_t stream) {
-  plan_kernel<<<1, 1024, 0, stream>>>(prm.seqlens, prm.nrb, prm.n_items, prefix_out, prm.status);
+  plan_kernel<<<1, 1024, 0, stream>>>(prm.seqlens, prm.nrb, prm.n_items, prm.tile_keys, prm.ovh, prefix_out, prm.status);
   return cudaGetLastError();
 }
 
 cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream) {
   const int warps_per_block = 4;   // small blocks: one fits beside a decode CTA (registers), so part of the grid is resident before the decode kernel ends
-  const long rows = static_cast<long>(prm.B) * prm.nrb * kRowBlock;
+  const long rows = static_cast<long>(prm.B) * prm.nrb * prm.item_rows;
   const int blocks = static_cast<int>((rows + warps_per_block - 1) / warps_per_block);
   // programmatic dependent launch: the blocks may be placed while the decode kernel drains; they wait inside
   cudaLaunchConfig_t cfg = {};

@@ -77,32 +77,26 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legiti
 // Slow path of a wait, kept out of line so that the many call sites stay small (the role loops are
 // executed by single warps and are sensitive to instruction-cache footprint).
 template <bool kClusterAcquire>
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
   const uint64_t t0 = global_timer_ns();
   while (true) {
     for (int i = 0; i < 256; ++i) {
       if (kClusterAcquire ? mbar_test_cluster_acquire(bar, parity) : mbar_test(bar, parity)) return true;
     }
-    if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+    if (global_timer_ns() - t0 > limit_ns) return false;
   }
 }
 
-// Waits for the phase with the given parity to complete; false after kWaitLimitNs.
+// Waits for the phase with the given parity to complete; false after limit_ns (kWaitLimitNs unless stated).
 template <bool kClusterAcquire = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
   if (kClusterAcquire ? mbar_test_cluster_acquire(bar, parity) : mbar_test(bar, parity)) return true;
-  return mbar_wait_slow<kClusterAcquire>(bar, parity);
+  return mbar_wait_slow<kClusterAcquire>(bar, parity, limit_ns);
 }
 
 // ------------------------------------------------------------------ fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async_all() {
-  asm volatile("fence.proxy.async;" ::: "memory");
-}
-__device__ __forceinline__ void fence_acq_rel_cluster() {
-  asm volatile("fence.acq_rel.cluster;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_before_sync() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -128,9 +122,6 @@ __device__ __forceinline__ void cluster_arrive() {
 __device__ __forceinline__ void cluster_wait() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 __device__ __forceinline__ void st_cluster_b32(uint32_t cluster_addr, uint32_t a) {
   asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(cluster_addr), "r"(a) : "memory");
 }
@@ -139,15 +130,8 @@ __device__ __forceinline__ void st_cluster_b32(uint32_t cluster_addr, uint32_t a
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
-// 2-D tiled load global -> this CTA's shared memory; completion is counted in bytes on `bar`.
-// x (innermost coordinate, elements) times the element size must be a multiple of 16 bytes.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tmap, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-
+// Tiled loads global -> this CTA's shared memory; completion is counted in bytes on `bar`.  The innermost
+// coordinate times the element size must be a multiple of 16 bytes.
 // 3-D tiled load (innermost coordinate first).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const void* tmap, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -162,19 +146,20 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tmap,
       ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
-// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster; the bytes are
-// counted on a barrier of the destination CTA.  Both addresses 16-byte aligned, size a multiple of 16.
-// Earlier generic-proxy writes to the source need fence.proxy.async first.
-__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t cluster_bar) {
+// The same loads issued by one CTA of an MMA pair (cluster ranks 2k, 2k+1): the data lands in this CTA's shared
+// memory, the bytes are counted on `cluster_bar`, which may be a barrier of the other CTA of the pair (an address
+// from map_to_cta) -- the pair's MMA issuer waits on one barrier for both halves of an operand.  No multicast.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst_smem, const void* tmap, int x, int y, int z, uint32_t cluster_bar) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(cluster_bar)
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(cluster_bar)
       : "memory");
 }
-// Brings a tile into L2 without a shared-memory destination.
-__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-               ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y) : "memory");
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst_smem, const void* tmap, int c0, int c1, int c2, int c3, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(cluster_bar)
+      : "memory");
 }
 // 256-bit read-only global load (32-byte aligned address).
 __device__ __forceinline__ void ldg_256(const void* p, uint32_t (&r)[32], int at) {
@@ -207,6 +192,17 @@ __device__ __forceinline__ void tmem_relinquish() {
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// The pair forms (one warp with the same index in each CTA of an MMA pair executes them): a kernel that issues
+// cta_group::2 MMAs allocates, relinquishes and frees with cta_group::2 as well.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -243,20 +239,11 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
 //   bits  0..13 start address >> 4      bits 16..29 leading-dimension byte offset >> 4
 //   bits 32..45 stride byte offset >> 4 bits 46..47 descriptor version (1 on sm_100)
 //   bits 61..63 swizzle mode (2 = 128 B)
+// The descriptor is handled as two 32-bit halves (smem_desc_lo / smem_desc_hi_sw128 below).
 // K-major operand (rows = M or N index, 64 bf16 of K per 128-byte row): rows of an 8-row group are
 // 128 B apart, groups are `sbo` bytes apart; the leading offset is not used.
 // MN-major operand (rows = K index, 64 bf16 of M/N per 128-byte row): `lbo` is the distance between
 // successive 64-element blocks along M/N, `sbo` between successive groups of 8 K-rows.
-__device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-
 // The same descriptor split in halves: only the low word depends on the address, so an issue loop can
 // keep the high word and step the low word by (byte offset >> 4).
 __host__ __device__ constexpr uint32_t smem_desc_hi_sw128(uint32_t sbo_bytes) {
@@ -308,6 +295,33 @@ __device__ __forceinline__ void mma_commit_multicast(uint32_t bar, uint16_t cta_
                ::"r"(bar), "h"(cta_mask) : "memory");
 }
 
+// ---- MMAs over a pair of CTAs (cluster ranks 2k and 2k+1), issued by one thread of the even one.  M = 256: each
+// CTA contributes its own 128 rows of A (same tensor-memory address / same shared-memory offset in both) and
+// receives its 128 rows of D in its own tensor memory; B (N x 16) is split, the even CTA holding rows 0..N/2-1 of
+// it and the odd CTA rows N/2..N-1 at the same shared-memory offset.
+__device__ __forceinline__ void mma_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// One arrival on the barrier at this shared-memory offset in every CTA of cta_mask once all pair MMAs issued so
+// far by this thread have completed (in both CTAs of the pair).
+__device__ __forceinline__ void mma_commit_pair_multicast(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(cta_mask) : "memory");
+}
+
 // Asynchronous stores into the shared memory of a CTA of the cluster; each adds its size to the transaction
 // count of a barrier of that CTA.  Generic-proxy writes: a consumer that reads them through the async proxy
 // (TMA, tcgen05.mma) fences with fence.proxy.async after its wait.
@@ -315,11 +329,6 @@ __device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, uint32_t a, u
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
                ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(cluster_bar) : "memory");
 }
-__device__ __forceinline__ void st_async_b32(uint32_t cluster_addr, uint32_t a, uint32_t cluster_bar) {
-  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
-               ::"r"(cluster_addr), "r"(a), "r"(cluster_bar) : "memory");
-}
-
 // Byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled tile whose rows are 128 B
 // (the pattern TMA's SWIZZLE_128B produces and the descriptors above expect; the tile base must be
 // 1024-byte aligned): chunk index XOR (row mod 8).
@@ -346,12 +355,6 @@ __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-
 // max of three (one instruction on sm_100).
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float r;

@@ -12,11 +12,11 @@
 #include "../../include/amla.h"
 #include "amla_common.cuh"
 
+#include <mutex>
+
 namespace amla {
-cudaError_t launch_plan(const DecodeParams& prm, int* prefix_out, cudaStream_t stream);
-cudaError_t launch_combine(const DecodeParams& prm, cudaStream_t stream);
-cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* unsupported);
-int decode_tc_parts(int sm_count);
+int configure_schedule(DecodeParams& prm, int device, int sms, int flags);
+int launch_decode_call(const DecodeParams& prm, int* prefix, cudaStream_t stream, int* launches, void (*mark)(int, cudaStream_t));
 }  // namespace amla
 
 namespace {
@@ -42,6 +42,7 @@ static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
 struct PerDevice {
   std::atomic<int> ready{0};
+  std::mutex setup;               // serialises the one-time lookup when first calls race on a device
   unsigned char* scratch = nullptr;
   int sms = 0;
   int cc_major = 0;
@@ -53,6 +54,8 @@ int setup_device(int device, PerDevice** out) {
   if (device < 0 || device >= 64) return AMLA_ERR_INVALID_ARG;
   PerDevice& d = g_dev[device];
   if (!d.ready.load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(d.setup);
+    if (d.ready.load(std::memory_order_acquire)) { *out = &d; return AMLA_OK; }
     void* p = nullptr;
     int sms = 0, cc = 0;
     if (cudaGetSymbolAddress(&p, g_scratch) != cudaSuccess || p == nullptr ||
@@ -86,8 +89,8 @@ extern "C" int amla_mla_decode_static(const void* q, const void* kv_cache, const
     return AMLA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(block_table) | reinterpret_cast<uintptr_t>(seqlens) | reinterpret_cast<uintptr_t>(lse)) & 3)
     return AMLA_ERR_INVALID_ARG;
-  const int nrb = (Sq * H + kRowBlock - 1) / kRowBlock;
-  const long long n_items = static_cast<long long>(B) * nrb;
+  // counted in 128-row blocks, whichever kernel the shape selects
+  const long long n_items = static_cast<long long>(B) * ((Sq * H + kRowBlock - 1) / kRowBlock);
   if (n_items > kMaxItems) return AMLA_ERR_STATIC_LIMIT;      // more (sequence, row block) pairs than the scratch has room for
 
   int device = 0;
@@ -96,8 +99,7 @@ extern "C" int amla_mla_decode_static(const void* q, const void* kv_cache, const
   const int rc = setup_device(device, &dev);
   if (rc != AMLA_OK) return rc;
   if (dev->cc_major != 10) return AMLA_ERR_UNSUPPORTED;
-  const int parts = decode_tc_parts(dev->sms);
-  if (parts > kMaxParts) return AMLA_ERR_STATIC_LIMIT;       // a device with more SMs than the scratch was sized for
+  if (dev->sms > AMLA_STATIC_MAX_SMS) return AMLA_ERR_STATIC_LIMIT;   // a device with more SMs than the scratch was sized for
 
   unsigned char* ws = dev->scratch;
   DecodeParams prm;
@@ -116,25 +118,32 @@ extern "C" int amla_mla_decode_static(const void* q, const void* kv_cache, const
   prm.scale_log2 = softmax_scale * kLog2e;
   prm.B = B; prm.Sq = Sq; prm.H = H;
   prm.R = Sq * H;
-  prm.nrb = nrb;
-  prm.n_items = static_cast<int>(n_items);
   prm.num_blocks = num_blocks;
   prm.max_blocks_per_seq = max_blocks_per_seq;
   prm.flags = AMLA_RESCALE_ALG2 | AMLA_LAZY(AMLA_DEFAULT_TAU);
   prm.tau = static_cast<float>(AMLA_DEFAULT_TAU);
-  prm.P = parts;
+  const int rcfg = configure_schedule(prm, device, dev->sms, prm.flags);
+  if (rcfg != AMLA_OK) return rcfg;
 
   // Nothing in the scratch has to be cleared by the host: the first kernel (the schedule kernel, or for few items the
-  // decode kernel itself) rewrites the status word and the whole
-  // prefix, and every partial that the combine reads is written by the decode kernel of the same call.
+  // decode kernel itself) rewrites the status word and the whole prefix, and every partial that the combine reads is
+  // written by the decode kernel of the same call.
+  int launches = 0;
+  return launch_decode_call(prm, prefix, static_cast<cudaStream_t>(cuda_stream), &launches, nullptr);
+}
+
+extern "C" int amla_static_check_status(void* cuda_stream) {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  PerDevice* dev = nullptr;
+  const int rc = setup_device(device, &dev);
+  if (rc != AMLA_OK) return rc;
+  int st = 0;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  prm.fused_plan = prm.n_items <= kFusedPlanMaxItems ? 1 : 0;
-  if (!prm.fused_plan && launch_plan(prm, prefix, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-  int unsupported = 0;
-  if (launch_decode_tc(prm, stream, &unsupported) != cudaSuccess) {
+  if (cudaMemcpyAsync(&st, dev->scratch + kStatusOff, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
     cudaGetLastError();
-    return unsupported ? AMLA_ERR_UNSUPPORTED : AMLA_ERR_CUDA;
+    return AMLA_ERR_CUDA;
   }
-  if (launch_combine(prm, stream) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
-  return AMLA_OK;
+  return st == amla::kStatusOk ? AMLA_OK : AMLA_ERR_DEVICE_TIMEOUT;
 }

@@ -10,7 +10,12 @@ import pytest
 from paper_2509_25224_b200 import binding, build, synth
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-UNIT_OVERHEAD = 10      # kUnitOverheadTiles of the schedule
+
+
+def _variant(Sq, H):
+    """(rows per item, keys per tile, overhead positions) of the schedule for a shape: up to 128 query rows per
+    sequence the items are 128-row blocks with one-page tiles, above that 256-row blocks with two-page tiles."""
+    return (256, 128, 5) if Sq * H > 128 else (128, 64, 10)
 
 
 @pytest.fixture(scope="module")
@@ -34,8 +39,8 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_status_strings(lib):
     assert binding.status_string(0) == "ok"
-    seen = {binding.status_string(c) for c in range(-5, 1)}
-    assert len(seen) == 6 and "unknown status" not in seen
+    seen = {binding.status_string(c) for c in range(-6, 1)}
+    assert len(seen) == 7 and "unknown status" not in seen
     assert binding.status_string(-99) == "unknown status"
 
 
@@ -57,9 +62,10 @@ def test_null_and_bad_arguments_are_rejected_before_any_cuda_call(lib):
 
 def _check_plan(seqlens, Sq, H, P):
     units = binding.plan_host(seqlens, Sq, H, P)
-    nrb = (Sq * H + 127) // 128
+    item_rows, tile_keys, UNIT_OVERHEAD = _variant(Sq, H)
+    nrb = (Sq * H + item_rows - 1) // item_rows
     n_items = len(seqlens) * nrb
-    tiles = [(max(int(seqlens[it // nrb]), 0) + 63) // 64 for it in range(n_items)]
+    tiles = [(max(int(seqlens[it // nrb]), 0) + tile_keys - 1) // tile_keys for it in range(n_items)]
     cover = [np.zeros(t, dtype=np.int32) for t in tiles]
     per_part = np.zeros(P, dtype=np.int64)
     slots = set()
@@ -118,6 +124,36 @@ def test_plan_small_case_by_hand(lib):
     # the first item, part 1 = [7,14) the second
     u = binding.plan_host(np.array([129, 10]), 1, 128, 2)
     assert u.tolist() == [[0, 0, 0, 3, -1, 1], [1, 1, 0, 1, -1, 1]]
+
+
+def test_plan_small_case_by_hand_256_row_items(lib):
+    # Sq = 2, H = 128: one 256-row item per sequence, 128-key tiles, 5 overhead positions.  Lengths 300 and 100 give
+    # 3 and 1 tiles: positions [tiles 0-2 | 5 overhead, tile 0] = 9; 3 parts own [0,3), [3,6), [6,9): the first
+    # item is one unit of part 0, the second item's tile (position 8) falls into part 2
+    u = binding.plan_host(np.array([300, 100]), 2, 128, 3)
+    assert u.tolist() == [[0, 0, 0, 3, -1, 1], [2, 1, 0, 1, -1, 1]]
+    # Sq = 3: 384 rows are two 256-row items per sequence (the second half filled)
+    u = binding.plan_host(np.array([128]), 3, 128, 1)
+    assert u.tolist() == [[0, 0, 0, 1, -1, 1], [0, 1, 0, 1, -1, 1]]
+
+
+def test_paging_validation_names_the_bad_entry(lib):
+    bt = np.array([[3, 1, -1], [0, 2, 7]], dtype=np.int32)
+    assert binding.validate_paging_host(bt, [100, 192], 8) is None            # unused entries are ignored
+    assert binding.validate_paging_host(bt, [129, 192], 8) == (0, 2)          # third page of sequence 0 is -1
+    assert binding.validate_paging_host(bt, [100, 192], 7) == (1, 2)          # page 7 of a 7-page cache
+    assert binding.validate_paging_host(bt, [100, 193], 8) == (1, -1)         # longer than the table allows
+    assert binding.validate_paging_host(bt, [-1, 0], 8) == (0, -1)
+    z = ctypes.c_void_p(0)
+    assert lib.amla_validate_paging_host(z, z, 1, 1, 1, None, None) == -1
+
+
+def test_wait_selftest_rejects_bad_arguments_without_a_device(lib):
+    z = ctypes.c_void_p(0)
+    assert lib.amla_wait_selftest(z, 1000, z) == -1
+    assert lib.amla_wait_selftest(ctypes.c_void_p(256), 0, z) == -1
+    assert lib.amla_wait_selftest(ctypes.c_void_p(256), 10**9, z) == -1       # limits above 0.1 s are refused
+    assert lib.amla_wait_selftest(ctypes.c_void_p(258), 1000, z) == -1
 
 
 def test_batch_sharding_partitions_sequences():

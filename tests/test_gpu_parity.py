@@ -40,6 +40,45 @@ def test_head_and_token_shapes(Sq, H):
     check_full(w)
 
 
+@pytest.mark.parametrize("lens", [[1], [64], [65], [128], [129], [191], [192], [193], [1000, 3, 0, 257, 64]])
+def test_256_row_kernel_tile_tails(lens):
+    # more than 128 query rows per sequence: 256-row items, 128-key tiles whose second page may be absent or partial
+    w = synth.make_workload("q", len(lens), 2, 128, lens, seed=400 + sum(lens))
+    check_full(w)
+    check_full(w, binding.RESCALE_ALG2 | binding.lazy(0))
+
+
+def test_256_row_kernel_against_128_row_blocks():
+    # the same problem through both kernels (256-row items vs independent 128-row blocks): both meet the oracle
+    w = synth.make_workload("ab", 3, 2, 128, [5000, 777, 2049], seed=431)
+    for flags in (binding.DEFAULT_FLAGS, binding.DEFAULT_FLAGS | binding.FLAG_KERNEL_ROWS128):
+        check_full(w, flags)
+    w = synth.make_workload("ab4", 2, 4, 128, [3000, 130], seed=432)
+    for flags in (binding.DEFAULT_FLAGS, binding.DEFAULT_FLAGS | binding.FLAG_KERNEL_ROWS128):
+        check_full(w, flags)
+
+
+def test_unguarded_add_on_zero_free_inputs():
+    # the literal single integer add of Algorithm 2 line 14 (no guard for zeros): valid when no accumulator is
+    # exactly zero or tiny, which N(0,1) inputs ensure
+    for Sq in (1, 2):
+        w = synth.make_workload("ung", 2, Sq, 128, [3000, 1500], seed=440 + Sq)
+        for mode in (binding.RESCALE_ALG2, binding.RESCALE_FOLD):
+            check_full(w, mode | binding.lazy(0) | binding.FLAG_UNGUARDED_ADD)
+
+
+def test_bounded_wait_reports_a_timeout_instead_of_hanging():
+    import torch
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    binding.check_status(ws)
+    binding.wait_selftest(ws, limit_ns=1_000_000)        # waits 1 ms on a barrier nothing arrives on
+    with pytest.raises(binding.AmlaError) as e:
+        binding.check_status(ws)
+    assert e.value.code == -5
+    # the context is intact and a decode on a workspace resets its status word
+    check_full(synth.config_tiny())
+
+
 def test_all_sequences_empty():
     w = synth.make_workload("e", 3, 2, 128, [0, 0, 0], seed=7)
     out, lse, _ = run_gpu(w)
@@ -49,6 +88,16 @@ def test_all_sequences_empty():
 def test_many_short_sequences_more_items_than_parts():
     rng = np.random.default_rng(9)
     w = synth.make_workload("m", 200, 1, 128, rng.integers(0, 200, 200), seed=8)
+    check_full(w)
+
+
+def test_hundreds_of_one_page_units_per_cluster():
+    # 640 sequences of 1..64 keys: every cluster runs through many one-page units back to back, so the softmax of a
+    # later unit can be far ahead of the epilogue of an earlier one (the hand-off of the final scalars must hold it back)
+    rng = np.random.default_rng(21)
+    w = synth.make_workload("short", 640, 1, 128, rng.integers(1, 65, 640), seed=22)
+    check_full(w)
+    w = synth.make_workload("short2", 300, 2, 128, rng.integers(1, 130, 300), seed=23)
     check_full(w)
 
 
