@@ -66,7 +66,21 @@ constexpr uint32_t kBarBytes = 512;
 constexpr int kSmemPlanItems = 128;
 constexpr uint32_t kOffPlan = kOffBars + kBarBytes;
 constexpr uint32_t kOffSeqlens = kOffPlan + ((kSmemPlanItems + 1) * 4 + 15) / 16 * 16;
+#ifdef AMLA_TRACE
+// trace builds: every CTA keeps its stamps (low 32 bits of its SM's cycle counter) in shared memory, so that taking
+// one does not put a global store in front of the role's next release, and dumps them when it is done
+constexpr int kQTraceEvents = 16, kQTraceIdx = 128;
+constexpr uint32_t kOffTrace = kOffSeqlens + kSmemPlanItems * 4;
+constexpr uint32_t kSmemBytes = kOffTrace + kQTraceEvents * kQTraceIdx * 4;
+#define QSTAMP(smem_base_, ev, idx)                                                                          \
+  do {                                                                                                       \
+    if (static_cast<unsigned>(idx) < static_cast<unsigned>(kQTraceIdx))                                      \
+      st_shared_b32((smem_base_) + kOffTrace + ((ev) * kQTraceIdx + (idx)) * 4, static_cast<uint32_t>(clock64())); \
+  } while (0)
+#else
 constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
+#define QSTAMP(smem_base_, ev, idx) do { } while (0)
+#endif
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
 static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0 && kOffStage % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
@@ -76,17 +90,19 @@ constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 column
 
 constexpr uint16_t kMaskScore = 0x3, kMaskValue = 0xC, kMaskAll = 0xF;
 
-// X_PV exists in all four CTAs: PVDONE in the value CTAs, "P buffer free" in the score CTAs.  Barriers marked (L)
-// are used in the pair's even CTA only; the odd CTA's warps arrive on them remotely.
+// X_PV exists in all four CTAs: PVDONE in the value CTAs, "P buffer free" in the score CTAs.  Barriers marked (R)
+// gather warps of both CTAs of a pair for the MMA issuer in the even CTA: the warps of either CTA arrive on their
+// own CTA's copy (a remote arrival with cluster-scope release stalls the arriving thread for thousands of cycles),
+// and in the odd CTA the otherwise idle warp 5 relays each completed phase as ONE arrival on the even CTA's copy.
 enum { X_PV = 0, X_COMMON = X_PV + kNumP };
-enum { A_KFULL = X_COMMON /*L*/, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2 /*L*/,
-       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2 /*L*/, A_QFREE, A_NUM };
-enum { B_VFULL = X_COMMON /*L*/, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP /*L*/,
+enum { A_KFULL = X_COMMON /* even CTA */, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2 /*R*/,
+       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2 /*R*/, A_QFREE, A_NUM };
+enum { B_VFULL = X_COMMON /* even CTA */, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP /*R*/,
        B_NUM = B_OREADY + kNumP };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
 
 struct Unit {
-  int b, r0, n_b, t0, t1, slot;    // r0: first row of the 256-row block; t0, t1: 128-key tiles
+  int b, r0, n_b, t0, t1, it;      // r0: first row of the 256-row block; t0, t1: 128-key tiles; it: item index
 };
 
 struct UnitIter {
@@ -110,13 +126,17 @@ struct UnitIter {
       g = min(e, g1);
       if (hi > lo) { u.t0 = lo - a; u.t1 = hi - a; break; }
     }
+    u.it = it;
     u.b = it / prm.nrb;
     u.r0 = (it % prm.nrb) * kItemRows;
     u.n_b = min(max(seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
-    int p_first, p_last;
-    const int nsplit = plan.item_parts(it, &p_first, &p_last);
-    u.slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
     return true;
+  }
+  // Partial slot of the unit, -1 if its item lies in one part (several divisions: only the epilogue asks)
+  __device__ int slot_of(const Unit& u) const {
+    int p_first, p_last;
+    const int nsplit = plan.item_parts(u.it, &p_first, &p_last);
+    return nsplit == 1 ? -1 : plan.slot_of(p, u.it, p_first);
   }
 };
 
@@ -141,10 +161,10 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
   return __all_sync(0xffffffffu, mbar_wait<kClusterAcquire>(bar, parity));
 }
 
-// One arrival per warp on a barrier of the pair's even CTA, after every lane's preceding work.
-__device__ __forceinline__ void warp_arrive_cluster(uint32_t cluster_bar, int lane) {
+// One arrival per warp on a barrier of this CTA, after every lane's preceding work.
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
   __syncwarp();
-  if (lane == 0) mbar_arrive_cluster(cluster_bar);
+  if (lane == 0) mbar_arrive(bar);
 }
 
 __device__ __forceinline__ void prefetch_q_row(const DecodeParams& prm, const Unit& u, int row) {
@@ -176,8 +196,9 @@ __device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int
 }
 
 struct RoleCtx {
-  uint32_t smem_base, bars, tbase, lead_bars;   // lead_bars: barrier area of the pair's even CTA (cluster address)
+  uint32_t smem_base, bars, tbase;
   int half, tid;                                // half: which 128 rows of the 256-row block this CTA owns
+  int part;
 };
 
 // The softmax warpgroup's work on one unit: its 128-key score tiles; the final scalars travel with the last page.
@@ -203,6 +224,7 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
     ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
     if (!ok) break;
     tc_fence_after_sync();
+    if (tid == 0) QSTAMP(c.smem_base, 2, gs);
     const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
     const int nvis = visible - t * kTileKeys;            // keys of this tile the row sees (may be <= 0)
     const bool last_tile = t + 1 == u.t1;
@@ -245,6 +267,7 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
       ext = scale_nn ? fmaxf(ext, ext_b) : fminf(ext, ext_b);
       const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
       const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
+      if (tid == 0) QSTAMP(c.smem_base, 13, gs);
       // Line 10's factor S16 goes into the exponential's argument (the remark after Algorithm 2).  The row sum of
       // line 6 is the sum of the same FP32 values, taken before the bf16 cast and divided by S16 once per tile.
       const float nsub = log2f_approx(sp.p_scale) - sp.m2_sub;
@@ -285,7 +308,8 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           tmem_ld_32x32b_x32(scol + 64, b0);
         } else {                       // the score tile has been read for the last time
           tc_fence_before_sync();
-          warp_arrive_cluster(c.lead_bars + 8u * (A_SEMPTY + sb), lane);
+          warp_arrive(bar(A_SEMPTY + sb), lane);
+          if (tid == 0) QSTAMP(c.smem_base, 3, gs);
         }
         // One staging buffer: the copy warps of the previous page must have read it into registers.  The barrier
         // is probed ahead of the last chunk's arithmetic, so that the probe's latency is not exposed.
@@ -294,6 +318,7 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
         const uint32_t s2 = gt & 1;
         if (!__all_sync(0xffffffffu, stage_free)) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
         if (!ok) break;
+        if (tid == 0) QSTAMP(c.smem_base, 14, gt);
         const uint32_t stg = smem_base + kOffStage;
 #pragma unroll
         for (int cc = 0; cc < 8; ++cc)
@@ -315,6 +340,7 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           }
         }
         mbar_arrive(bar(A_PSTAGED + s2));
+        if (tid == 0) QSTAMP(c.smem_base, 4, gt);
         ++gt;
       }
     };
@@ -322,6 +348,29 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
     else tile_body(std::false_type{});
   }
   return (static_cast<uint64_t>(gt) << 32) | (static_cast<uint64_t>(gs) << 1) | (ok ? 1u : 0u);
+}
+
+// Relay warp of a pair's odd CTA: lane l < n_lanes watches barrier `first + l` of this CTA and passes each of its
+// `phases` completed phases on as one arrival on the same barrier of the even CTA.  The lanes poll without blocking
+// and in lockstep (a blocking wait in one lane of a diverged warp holds the other lanes back for its whole
+// suspension time).  Returns false if a phase did not come within the wait limit.
+template <bool kProxyFence>
+__device__ __forceinline__ bool relay_phases(uint32_t bars, uint32_t lead_bars, int first, int lane, int phases) {
+  const uint32_t lb = bars + 8u * (first + lane), rb = lead_bars + 8u * (first + lane);
+  int k = 0;
+  uint64_t t_start = global_timer_ns();
+  for (uint32_t spin = 0;; ++spin) {
+    bool progress = false;
+    if (k < phases && mbar_probe(lb, k & 1)) {
+      if (kProxyFence) fence_proxy_async_smem();
+      mbar_arrive_cluster_relaxed(rb);
+      ++k;
+      progress = true;
+    }
+    if (__all_sync(0xffffffffu, k >= phases)) return true;
+    if (__any_sync(0xffffffffu, progress)) t_start = global_timer_ns(); else __nanosleep(32);
+    if ((spin & 1023u) == 1023u && __any_sync(0xffffffffu, global_timer_ns() - t_start > kWaitLimitNs)) return false;
+  }
 }
 
 }  // namespace
@@ -354,14 +403,14 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     if (is_score) {
       for (int i = 0; i < kNumKSlots; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
       for (int i = 0; i < 2; ++i) {
-        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 8);         // 4 softmax warps of either CTA
+        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), leader ? 5 : 4);   // 4 softmax warps (+ the odd CTA's relay)
         mbar_init(bar(A_PSTAGED + i), 128); mbar_init(bar(A_STAGEFREE + i), 2);
       }
-      mbar_init(bar(A_QREADY), 16);                                              // 8 loading warps of either CTA
+      mbar_init(bar(A_QREADY), leader ? 9 : 8);                                         // 8 loading warps (+ relay)
       mbar_init(bar(A_QFREE), 1);
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
-      for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 16); }   // 8 correction warps of either CTA
+      for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), leader ? 9 : 8); }   // 8 correction warps (+ relay)
     }
     fence_mbar_init();
     prefetch_tensormap(&k_map);
@@ -374,9 +423,15 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
   cluster_wait();
   tc_fence_after_sync();
   const uint32_t tbase = ld_shared_b32(tmem_slot);
+#ifdef AMLA_TRACE
+  for (int i = tid; i < kQTraceEvents * kQTraceIdx; i += kThreads) st_shared_b32(smem_base + kOffTrace + 4 * i, 0u);
+  __syncthreads();
+#endif
 
+  if (tid == 0) QSTAMP(smem_base, 15, 1);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
+  if (tid == 0) QSTAMP(smem_base, 15, 2);
   const int* prefix = prm.prefix;
   const int* seqlens = prm.seqlens;
   if (prm.fused_plan) {
@@ -417,6 +472,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     if (first.next(fu)) prefetch_q_row(prm, fu, half * kRowBlock + tid);
   }
 
+  if (tid == 0) QSTAMP(smem_base, 15, 3);
   bool ok = true;
   UnitIter iter(prm, prefix, seqlens, part);
   Unit u;
@@ -430,11 +486,12 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       // ---- softmax warpgroup: thread = query row
       const int r = tid;
       const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
-      const RoleCtx ctx{smem_base, bars, tbase, lead_bars, half, tid};
+      const RoleCtx ctx{smem_base, bars, tbase, half, tid, part};
       while (ok && iter.next(u)) {
         ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);      // the previous unit's QK^T is finished with Q
         if (!ok) break;
         tc_fence_after_sync();
+        if (tid == 0) QSTAMP(smem_base, 15, 8 + 4 * un);
         {
           const int row = u.r0 + half * kRowBlock + r;
           const bool valid = row < prm.R;
@@ -443,7 +500,8 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           tmem_wait_st();
         }
         tc_fence_before_sync();
-        warp_arrive_cluster(lead_bars + 8u * A_QREADY, lane);
+        warp_arrive(bar(A_QREADY), lane);
+        if (tid == 0) QSTAMP(smem_base, 15, 9 + 4 * un);
         const uint64_t ret = softmax_unit<kMode>(prm, ctx, u, gt, gs);
         gt = static_cast<uint32_t>(ret >> 32);
         gs = static_cast<uint32_t>(ret & 0xffffffffu) >> 1;
@@ -518,11 +576,24 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             ok = mbar_wait<true>(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
+            QSTAMP(smem_base, 0, gs);
             const uint32_t d = tbase + kSCol + 128 * sb;
+            // the three slots of the tile are probed together (their latencies overlap); the blocking wait runs
+            // only for one that is not there yet
+            bool have[3];
+            {
+              uint32_t s2 = slot, p2 = kpar;
+#pragma unroll
+              for (int gg = 0; gg < 3; ++gg) {
+                have[gg] = mbar_probe(bar(A_KFULL) + 8 * s2, p2);
+                if (++s2 == kNumKSlots) { s2 = 0; p2 ^= 1; }
+              }
+            }
 #pragma unroll
             for (int gg = 0; gg < 3; ++gg) {
-              ok = ok && mbar_wait<true>(bar(A_KFULL) + 8 * slot, kpar);
+              ok = ok && (have[gg] || mbar_wait<true>(bar(A_KFULL) + 8 * slot, kpar));
               if (ok) {
+                if (gg == 0) QSTAMP(smem_base, 12, gs);
                 const uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
 #pragma unroll
                 for (int cl = 0; cl < 3; ++cl) {
@@ -540,12 +611,22 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             }
             if (!ok) break;
             mma_commit_pair_multicast(bar(A_SFULL + sb), kMaskScore);
+            QSTAMP(smem_base, 1, gs);
           }
           if (!ok) break;
           mma_commit_pair_multicast(bar(A_QFREE), kMaskScore);
           ++un;
         }
         if (!ok) report_timeout(prm.status);
+      } else if (!leader) {
+        // ---- relay (odd CTA): lanes 0, 1 pass on the completed phases of SEMPTY[lane] (the tiles with that buffer),
+        // lane 2 those of QREADY (one per unit)
+        static_assert(A_QREADY == A_SEMPTY + 2 + 2 + 2, "lane 2 is moved onto QREADY below");
+        int n_units = 0, n_tiles = 0;
+        while (iter.next(u)) { ++n_units; n_tiles += u.t1 - u.t0; }
+        const int phases = lane == 2 ? n_units : lane < 2 ? (n_tiles + 1 - lane) / 2 : 0;
+        const int first = lane == 2 ? A_QREADY - 2 : A_SEMPTY;
+        if (!relay_phases<false>(bars, lead_bars, first, lane, phases) && lane == 0) report_timeout(prm.status);
       }
     } else if (wid >= 6 && wid < 6 + kNumCopyWarps) {
       // ---- copy warps: staged P~ / N (and, with a unit's last page, the final scalars) -> a free P buffer of this
@@ -572,7 +653,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           tmem_wait_st();
           fence_proxy_async_smem();
           tc_fence_before_sync();
-          warp_arrive_cluster(lead_bars + 8u * A_QREADY, lane);
+          warp_arrive(bar(A_QREADY), lane);
           ++un;
           UnitIter peek = iter;
           Unit nu;
@@ -599,7 +680,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           if (!ok) break;
           const uint32_t pfull = myV_bars + 8u * (B_PFULL + pb);
           const uint32_t dstp = myV_base + kOffP + pb * kPStride + (hv * kChunks * 32 + lane) * 16;
-          if (lane == 0 && hv == 0) mbar_arrive_expect_tx_cluster(pfull, last ? kPXferLast : kPXfer);
+          if (lane == 0 && hv == 0) { QSTAMP(smem_base, 5, gt); mbar_arrive_expect_tx_cluster(pfull, last ? kPXferLast : kPXfer); }
 #pragma unroll
           for (int i = 0; i < kChunks; ++i) {
             if (static_cast<int>(hv) * kChunks + i < nchunks) st_async_v4(dstp + i * 512, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
@@ -619,11 +700,13 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       const int c_first = partner ? 8 : 0;
       while (ok && iter.next(u)) {
         const int npages = 2 * (u.t1 - u.t0);
+        const int slot = partner ? -1 : iter.slot_of(u);
         float inv = 0.f, lse = 0.f;
         for (int pi = 0; pi < npages && ok; ++pi, ++gt) {
           const uint32_t s = gt % kNumP, k = gt / kNumP;
           ok = warp_wait<true>(bar(B_PFULL + s), k & 1);
           if (!ok) break;
+          if (tid == 0) QSTAMP(smem_base, 6, gt);
           const uint32_t pbuf = smem_base + kOffP + s * kPStride;
           const uint32_t nword = ld_shared_b32(pbuf + kNOff + r * 4);
           if (pi + 1 == npages && !partner) {
@@ -678,9 +761,8 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             tmem_wait_st();
             tc_fence_before_sync();
           }
-          // this CTA's P~ (remote asynchronous stores, generic proxy) is about to be read by the pair MMA
-          fence_proxy_async_smem();
-          warp_arrive_cluster(lead_bars + 8u * (B_OREADY + s), lane);
+          warp_arrive(bar(B_OREADY + s), lane);
+          if (tid == 0) QSTAMP(smem_base, 7, gt);
         }
         if (!ok) break;
         // ---- epilogue (line 20): out = O / (l * S16)
@@ -689,12 +771,13 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
           tc_fence_after_sync();
+          if (tid == 0) QSTAMP(smem_base, 15, 10 + 4 * un);
           const int row0 = u.r0 + half * kRowBlock;               // first row of this CTA within the sequence
           const bool valid = row0 + r < prm.R;
           const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
           const int rows_here = min(32, prm.R - row0 - wid * 32);
           __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + row0 + wid * 32) * kDv;
-          float* pbase = prm.part_o + (static_cast<size_t>(u.slot < 0 ? 0 : u.slot) * kItemRows + half * kRowBlock + wid * 32) * kDv;
+          float* pbase = prm.part_o + (static_cast<size_t>(slot < 0 ? 0 : slot) * kItemRows + half * kRowBlock + wid * 32) * kDv;
           uint32_t o[2][32];
           tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
 #pragma unroll 1
@@ -705,7 +788,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
               if (cq + e + 1 < 16) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (cq + e + 1), o[e ^ 1]);
               const int cc = cq + e;
               __syncwarp();
-              if (u.slot < 0) {
+              if (slot < 0) {
 #pragma unroll
                 for (int jj = 0; jj < 4; ++jj) {
                   const uint32_t w0 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 0]) * inv, __uint_as_float(o[e][8 * jj + 1]) * inv);
@@ -742,10 +825,11 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             }
           }
           if (valid) {
-            if (u.slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + row0 + r] = lse;
-            else prm.part_lse[static_cast<size_t>(u.slot) * kItemRows + half * kRowBlock + r] = lse;
+            if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + row0 + r] = lse;
+            else prm.part_lse[static_cast<size_t>(slot) * kItemRows + half * kRowBlock + r] = lse;
           }
           tc_fence_before_sync();
+          if (tid == 0) QSTAMP(smem_base, 15, 11 + 4 * un);
         }
         ++un;
       }
@@ -813,12 +897,15 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             const uint32_t s = gt % kNumP, k = gt / kNumP;
             ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
             if (!ok) break;
+            QSTAMP(smem_base, 10, gt);
             ok = mbar_wait<true>(bar(B_OREADY + s), k & 1);
             if (!ok) break;
+            QSTAMP(smem_base, 11, gt);
             tc_fence_after_sync();
             fence_proxy_async_smem();
             ok = mbar_wait<true>(bar(B_VFULL) + 8 * slot, vpar);
             if (!ok) break;
+            QSTAMP(smem_base, 8, gt);
             const uint32_t plo = plo0 + s * (kPStride >> 4);
             const uint32_t vlo = vlo0 + slot * (kVSlotBytes >> 4);
             const uint32_t acc0 = pi > 0 ? 1u : 0u;
@@ -832,18 +919,34 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             mma_commit_pair_multicast(bar(B_VEMPTY) + 8 * slot, kMaskValue);
             if (++slot == kNumVSlots) { slot = 0; vpar ^= 1; }
             mma_commit_pair_multicast(bar(X_PV + s), kMaskAll);   // PVDONE in the value CTAs, "P buffer free" in the score CTAs
+            QSTAMP(smem_base, 9, gt);
           }
           if (!ok) break;
         }
         if (!ok) report_timeout(prm.status);
+      } else if (!leader) {
+        // ---- relay (odd CTA): lane s passes on the completed phases of OREADY[s] (the pages in P buffer s).  The
+        // page's P~ in this CTA (remote asynchronous stores, generic proxy) is about to be read by the pair MMA.
+        int n_pages = 0;
+        while (iter.next(u)) n_pages += 2 * (u.t1 - u.t0);
+        const int phases = lane < kNumP ? (n_pages + kNumP - 1 - lane) / kNumP : 0;
+        if (!relay_phases<true>(bars, lead_bars, B_OREADY, lane, phases) && lane == 0) report_timeout(prm.status);
       }
     }
   }
 
   // teardown: nobody may still be writing into a CTA that has exited, and both CTAs of a pair must be done
   // with tensor memory before it is freed
+  if (tid == 0) QSTAMP(smem_base, 15, 4);
   tc_fence_before_sync();
   __syncthreads();
+  if (tid == 0) QSTAMP(smem_base, 15, 5);
+#ifdef AMLA_TRACE
+  if (prm.trace) {
+    for (int i = tid; i < kQTraceEvents * kQTraceIdx; i += kThreads)
+      prm.trace[static_cast<size_t>(blockIdx.x) * kQTraceEvents * kQTraceIdx + i] = ld_shared_b32(smem_base + kOffTrace + 4 * i);
+  }
+#endif
   cluster_arrive();
   cluster_wait();
   if (wid == 5) tmem_dealloc_pair(tbase, kTmemCols);

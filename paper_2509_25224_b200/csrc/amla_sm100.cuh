@@ -38,9 +38,15 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
-// Arrive on a barrier of another CTA of the cluster and add `bytes` to the transaction count it expects.
+// The same without the release: for a thread that only passes on an event it has itself observed as complete (the
+// release form makes the arriving thread wait for a cluster-scope fence, thousands of cycles under load).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// Arrive on a barrier of another CTA of the cluster and add `bytes` to the transaction count it expects.  Relaxed:
+// the arrival publishes nothing of its own -- the data are the asynchronous stores that complete the count.
 __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+  asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -329,6 +335,11 @@ __device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, uint32_t a, u
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
                ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(cluster_bar) : "memory");
 }
+__device__ __forceinline__ void st_async_v2(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];"
+               ::"r"(cluster_addr), "r"(a), "r"(b), "r"(cluster_bar) : "memory");
+}
+
 // Byte offset of element (row, 16-byte chunk) inside a 128-byte-swizzled tile whose rows are 128 B
 // (the pattern TMA's SWIZZLE_128B produces and the descriptors above expect; the tile base must be
 // 1024-byte aligned): chunk index XOR (row mod 8).
