@@ -77,9 +77,12 @@ constexpr uint32_t kSmemBytes = kOffTrace + kQTraceEvents * kQTraceIdx * 4;
     if (static_cast<unsigned>(idx) < static_cast<unsigned>(kQTraceIdx))                                      \
       st_shared_b32((smem_base_) + kOffTrace + ((ev) * kQTraceIdx + (idx)) * 4, static_cast<uint32_t>(clock64())); \
   } while (0)
+// event 15 holds wall-clock stamps (global timer, ns) of the kernel's phases, comparable across SMs and kernels
+#define QSTAMP_NS(smem_base_, idx) st_shared_b32((smem_base_) + kOffTrace + (15 * kQTraceIdx + (idx)) * 4, static_cast<uint32_t>(global_timer_ns()))
 #else
 constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
 #define QSTAMP(smem_base_, ev, idx) do { } while (0)
+#define QSTAMP_NS(smem_base_, idx) do { } while (0)
 #endif
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
 static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0 && kOffStage % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -225,6 +228,7 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
     if (!ok) break;
     tc_fence_after_sync();
     if (tid == 0) QSTAMP(c.smem_base, 2, gs);
+    if (tid == 0 && gs == 0) QSTAMP_NS(c.smem_base, 6);
     const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
     const int nvis = visible - t * kTileKeys;            // keys of this tile the row sees (may be <= 0)
     const bool last_tile = t + 1 == u.t1;
@@ -391,6 +395,12 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     return;
   }
 
+#ifdef AMLA_TRACE
+  const uint32_t t_entry = static_cast<uint32_t>(global_timer_ns());
+  for (int i = tid; i < kQTraceEvents * kQTraceIdx; i += kThreads) st_shared_b32(smem_base + kOffTrace + 4 * i, 0u);
+  __syncthreads();
+  if (tid == 0) st_shared_b32(smem_base + kOffTrace + (15 * kQTraceIdx + 0) * 4, t_entry);
+#endif
   const uint32_t bars = smem_base + kOffBars;
   auto bar = [&](int i) { return bars + 8u * i; };
   const uint32_t tmem_slot = bars + kBarBytes - 8;
@@ -423,15 +433,11 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
   cluster_wait();
   tc_fence_after_sync();
   const uint32_t tbase = ld_shared_b32(tmem_slot);
-#ifdef AMLA_TRACE
-  for (int i = tid; i < kQTraceEvents * kQTraceIdx; i += kThreads) st_shared_b32(smem_base + kOffTrace + 4 * i, 0u);
-  __syncthreads();
-#endif
 
-  if (tid == 0) QSTAMP(smem_base, 15, 1);
+  if (tid == 0) QSTAMP_NS(smem_base, 1);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
-  if (tid == 0) QSTAMP(smem_base, 15, 2);
+  if (tid == 0) QSTAMP_NS(smem_base, 2);
   const int* prefix = prm.prefix;
   const int* seqlens = prm.seqlens;
   if (prm.fused_plan) {
@@ -472,7 +478,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     if (first.next(fu)) prefetch_q_row(prm, fu, half * kRowBlock + tid);
   }
 
-  if (tid == 0) QSTAMP(smem_base, 15, 3);
+  if (tid == 0) QSTAMP_NS(smem_base, 3);
   bool ok = true;
   UnitIter iter(prm, prefix, seqlens, part);
   Unit u;
@@ -491,7 +497,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
         ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);      // the previous unit's QK^T is finished with Q
         if (!ok) break;
         tc_fence_after_sync();
-        if (tid == 0) QSTAMP(smem_base, 15, 8 + 4 * un);
+        if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 8 + 4 * un); };
         {
           const int row = u.r0 + half * kRowBlock + r;
           const bool valid = row < prm.R;
@@ -501,7 +507,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
         }
         tc_fence_before_sync();
         warp_arrive(bar(A_QREADY), lane);
-        if (tid == 0) QSTAMP(smem_base, 15, 9 + 4 * un);
+        if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 9 + 4 * un); };
         const uint64_t ret = softmax_unit<kMode>(prm, ctx, u, gt, gs);
         gt = static_cast<uint32_t>(ret >> 32);
         gs = static_cast<uint32_t>(ret & 0xffffffffu) >> 1;
@@ -771,7 +777,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
           tc_fence_after_sync();
-          if (tid == 0) QSTAMP(smem_base, 15, 10 + 4 * un);
+          if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 10 + 4 * un); };
           const int row0 = u.r0 + half * kRowBlock;               // first row of this CTA within the sequence
           const bool valid = row0 + r < prm.R;
           const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
@@ -829,7 +835,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             else prm.part_lse[static_cast<size_t>(slot) * kItemRows + half * kRowBlock + r] = lse;
           }
           tc_fence_before_sync();
-          if (tid == 0) QSTAMP(smem_base, 15, 11 + 4 * un);
+          if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 11 + 4 * un); };
         }
         ++un;
       }
@@ -937,10 +943,10 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
 
   // teardown: nobody may still be writing into a CTA that has exited, and both CTAs of a pair must be done
   // with tensor memory before it is freed
-  if (tid == 0) QSTAMP(smem_base, 15, 4);
+  if (tid == 0) QSTAMP_NS(smem_base, 4);
   tc_fence_before_sync();
   __syncthreads();
-  if (tid == 0) QSTAMP(smem_base, 15, 5);
+  if (tid == 0) QSTAMP_NS(smem_base, 5);
 #ifdef AMLA_TRACE
   if (prm.trace) {
     for (int i = tid; i < kQTraceEvents * kQTraceIdx; i += kThreads)
@@ -949,6 +955,9 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
 #endif
   cluster_arrive();
   cluster_wait();
+#ifdef AMLA_TRACE
+  if (prm.trace && tid == 0) prm.trace[static_cast<size_t>(blockIdx.x) * kQTraceEvents * kQTraceIdx + 15 * kQTraceIdx + 7] = static_cast<uint32_t>(global_timer_ns());
+#endif
   if (wid == 5) tmem_dealloc_pair(tbase, kTmemCols);
 }
 

@@ -91,7 +91,7 @@ enum { B_VFULL = X_COMMON, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY +
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
 
 struct Unit {
-  int b, r0, nrows, n_b, t0, t1, slot;
+  int b, r0, nrows, n_b, t0, t1, it;
 };
 
 // Walks the (part, item) intersections of this cluster's part in schedule order.
@@ -116,14 +116,18 @@ struct UnitIter {
       g = min(e, g1);
       if (hi > lo) { u.t0 = lo - a; u.t1 = hi - a; break; }   // else: only overhead positions of this item fell into the part
     }
+    u.it = it;
     u.b = it / prm.nrb;
     u.r0 = (it % prm.nrb) * kRowBlock;
     u.nrows = min(kRowBlock, prm.R - u.r0);
     u.n_b = min(max(seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
-    int p_first, p_last;
-    const int nsplit = plan.item_parts(it, &p_first, &p_last);
-    u.slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
     return true;
+  }
+  // Partial slot of the unit, -1 if its item lies in one part (several divisions: only the epilogue asks)
+  __device__ int slot_of(const Unit& u) const {
+    int p_first, p_last;
+    const int nsplit = plan.item_parts(u.it, &p_first, &p_last);
+    return nsplit == 1 ? -1 : plan.slot_of(p, u.it, p_first);
   }
 };
 
@@ -355,10 +359,11 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
       const bool live = st.l > 0.f;
       const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
       const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
+      // asynchronous remote stores counted on the barrier: no thread has to wait for a cluster-scope release
       const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;
-      st_cluster_b32(fdst, __float_as_uint(inv));
-      st_cluster_b32(fdst + 4, __float_as_uint(lse));
-      mbar_arrive_cluster(peerB_bars + 8u * (B_FINFULL + (un & 1)));
+      const uint32_t fbar = peerB_bars + 8u * (B_FINFULL + (un & 1));
+      if (tid == 0) mbar_arrive_expect_tx_cluster(fbar, 128 * 8);
+      st_async_v2(fdst, __float_as_uint(inv), __float_as_uint(lse), fbar);
     }
   }
   return (static_cast<uint64_t>(gt) << 32) | (static_cast<uint64_t>(gs) << 1) | (ok ? 1u : 0u);
@@ -402,7 +407,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
       for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 256); }
-      for (int i = 0; i < 2; ++i) mbar_init(bar(B_FINFULL + i), 128);
+      for (int i = 0; i < 2; ++i) mbar_init(bar(B_FINFULL + i), 1);    // one arrival that announces 128 x 8 bytes
     }
     fence_mbar_init();
     prefetch_tensormap(&kv_map);
@@ -719,6 +724,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
       const int c_first = partner ? 8 : 0;          // first of this warp's eight 32-column chunks
       while (ok && iter.next(u)) {
+        const int slot = partner ? -1 : iter.slot_of(u);
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
           const uint32_t s = gt % kNumP, k = gt / kNumP;
           ok = warp_wait<true>(bar(B_PFULL + s), k & 1);
@@ -796,7 +802,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             inv = __uint_as_float(x); lse = __uint_as_float(y);
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(peerA_bars + 8u * (A_FINFREE + (un & 1)));   // the entry may be rewritten
+          if (lane == 0) mbar_arrive_cluster_relaxed(peerA_bars + 8u * (A_FINFREE + (un & 1)));   // the entry may be rewritten
           const bool valid = r < u.nrows;
           // 32 columns at a time: each lane scales its row, the warp transposes the 32 x 32 tile through shared
           // memory (16-byte units XOR-swizzled by row), and writes whole 128-byte (FP32 partial) or 64-byte (bf16)
@@ -804,7 +810,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
           const int rows_here = min(32, u.nrows - wid * 32);          // valid rows of this warp's 32 (may be <= 0)
           __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + u.r0 + wid * 32) * kDv;
-          float* pbase = prm.part_o + (static_cast<size_t>(u.slot < 0 ? 0 : u.slot) * kRowBlock + wid * 32) * kDv;
+          float* pbase = prm.part_o + (static_cast<size_t>(slot < 0 ? 0 : slot) * kRowBlock + wid * 32) * kDv;
           uint32_t o[2][32];
           tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
 #pragma unroll 1
@@ -815,7 +821,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
               if (c + e + 1 < 16) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (c + e + 1), o[e ^ 1]);
               const int cc = c + e;
               __syncwarp();                                           // the tile is free again (previous read-back done)
-              if (u.slot < 0) {
+              if (slot < 0) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                   const uint32_t w0 = pack_bf16x2(__uint_as_float(o[e][8 * j + 0]) * inv, __uint_as_float(o[e][8 * j + 1]) * inv);
@@ -852,8 +858,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
             }
           }
           if (valid) {
-            if (u.slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
-            else prm.part_lse[static_cast<size_t>(u.slot) * kRowBlock + r] = lse;
+            if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
+            else prm.part_lse[static_cast<size_t>(slot) * kRowBlock + r] = lse;
           }
           tc_fence_before_sync();
           if (tid == 0) AMLA_STAMP(prm, part, 19, un);

@@ -50,7 +50,17 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
 // and are skipped; items without tiles get out = 0, lse = -inf; split items are merged:
 //   lse = ln sum_s exp(lse_s),  out = sum_s exp(lse_s - lse) * out_s.
 __global__ void combine_kernel(DecodeParams prm) {
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // launched early (programmatic dependent launch): the partials must be complete
+#ifdef AMLA_TRACE
+  unsigned long long t_ns;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
+  if (prm.trace && blockIdx.x == 0 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 0] = t_ns & 0xffffffffull;
+#endif
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef AMLA_TRACE
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
+  if (prm.trace && blockIdx.x == 0 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 1] = t_ns & 0xffffffffull;
+  if (prm.trace && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 2] = t_ns & 0xffffffffull;
+#endif   // launched early (programmatic dependent launch): the partials must be complete
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row_global = blockIdx.x * warps_per_block + (threadIdx.x >> 5);

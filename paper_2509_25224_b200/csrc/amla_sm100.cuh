@@ -34,12 +34,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Arrive on a barrier that lives in another CTA of the cluster (address from map_to_cta).
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-// The same without the release: for a thread that only passes on an event it has itself observed as complete (the
-// release form makes the arriving thread wait for a cluster-scope fence, thousands of cycles under load).
+// Arrive on a barrier that lives in another CTA of the cluster (address from map_to_cta), without a release: for a
+// thread that only passes on an event it has itself observed as complete.  (The release form makes the arriving
+// thread wait for a cluster-scope fence: thousands of cycles under load.)
 __device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_bar) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
@@ -127,9 +124,6 @@ __device__ __forceinline__ void cluster_arrive() {
 }
 __device__ __forceinline__ void cluster_wait() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void st_cluster_b32(uint32_t cluster_addr, uint32_t a) {
-  asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(cluster_addr), "r"(a) : "memory");
 }
 
 // ------------------------------------------------------------------ TMA
