@@ -26,14 +26,15 @@ constexpr int kMaxRows = 1024;   // Sq * H
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-  size_t status_off, prefix_off, part_lse_off, part_o_off, total;
+  size_t status_off, prefix_off, info_off, part_lse_off, part_o_off, total;
 };
 
 Layout make_layout(int n_items, int max_parts) {
   Layout l;
   l.status_off = 0;
   l.prefix_off = kAlign;
-  l.part_lse_off = l.prefix_off + align_up(sizeof(int) * (static_cast<size_t>(n_items) + 1));
+  l.info_off = l.prefix_off + align_up(sizeof(int) * (static_cast<size_t>(n_items) + 1));
+  l.part_lse_off = l.info_off + align_up(sizeof(int2) * static_cast<size_t>(n_items));
   l.part_o_off = l.part_lse_off + align_up(sizeof(float) * 2 * static_cast<size_t>(max_parts) * kRowBlock);
   l.total = l.part_o_off + sizeof(float) * 2 * static_cast<size_t>(max_parts) * kRowBlock * kDv;
   return l;
@@ -204,6 +205,7 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   prm.status = reinterpret_cast<int*>(ws + lay.status_off);
   int* prefix = reinterpret_cast<int*>(ws + lay.prefix_off);
   prm.prefix = prefix;
+  prm.item_info = reinterpret_cast<int2*>(ws + lay.info_off);
   prm.part_lse = reinterpret_cast<float*>(ws + lay.part_lse_off);
   prm.part_o = reinterpret_cast<float*>(ws + lay.part_o_off);
   prm.scale_log2 = softmax_scale * kLog2e;

@@ -30,6 +30,8 @@ struct DecodeParams {
   const int* prefix;             // [n_items + 1] linear tile index of each item's first tile
   float* part_o;                 // [2 * P, 128, 512] fp32 normalised partial outputs
   float* part_lse;               // [2 * P, 128]      partial lse (natural log)
+  int2* item_info;               // [n_items] (slot of the item's first partial, number of parts it is split over), written by
+                                 // the decode kernel for every item it touches, read by the combine
   float scale_log2;              // softmax_scale * log2(e)
   float tau;                     // lazy-reference threshold in octaves (0 = move the reference with every new maximum)
   int B, Sq, H;
@@ -149,6 +151,8 @@ struct Plan {
   __host__ __device__ int slot_of(int p, int it, int p_first) const {
     return 2 * p + ((p == p_first && prefix[it] > part_start(p)) ? 1 : 0);
   }
+  // The same from what item_info holds: slot of split s (0 = the part where the item begins) of an item
+  __host__ __device__ static int slot_of_split(int first_slot, int s) { return s == 0 ? first_slot : 2 * ((first_slot >> 1) + s); }
 };
 
 // ---------------------------------------------------------------------------------------------

@@ -135,10 +135,12 @@ struct UnitIter {
     u.n_b = min(max(seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
     return true;
   }
-  // Partial slot of the unit, -1 if its item lies in one part (several divisions: only the epilogue asks)
-  __device__ int slot_of(const Unit& u) const {
+  // Partial slot of the unit, -1 if its item lies in one part (several divisions: only the epilogue asks);
+  // *info = what the combine needs to know about the item
+  __device__ int slot_of(const Unit& u, int2* info) const {
     int p_first, p_last;
     const int nsplit = plan.item_parts(u.it, &p_first, &p_last);
+    *info = make_int2(plan.slot_of(p_first, u.it, p_first), nsplit);
     return nsplit == 1 ? -1 : plan.slot_of(p, u.it, p_first);
   }
 };
@@ -706,7 +708,9 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       const int c_first = partner ? 8 : 0;
       while (ok && iter.next(u)) {
         const int npages = 2 * (u.t1 - u.t0);
-        const int slot = partner ? -1 : iter.slot_of(u);
+        int2 info;
+        const int slot = partner ? -1 : iter.slot_of(u, &info);
+        if (tid == 0 && leader) prm.item_info[u.it] = info;
         float inv = 0.f, lse = 0.f;
         for (int pi = 0; pi < npages && ok; ++pi, ++gt) {
           const uint32_t s = gt % kNumP, k = gt / kNumP;

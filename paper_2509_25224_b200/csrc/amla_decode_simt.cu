@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
     int p_first, p_last;
     const int nsplit = plan.item_parts(it, &p_first, &p_last);
     const int slot = nsplit == 1 ? -1 : plan.slot_of(p, it, p_first);
+    if (tid == 0) prm.item_info[it] = make_int2(plan.slot_of(p_first, it, p_first), nsplit);
     const int32_t* bt = prm.block_table + static_cast<size_t>(b) * prm.max_blocks_per_seq;
 
     for (int pass = 0; pass * kRowsPerPass < nrows; ++pass) {

@@ -123,10 +123,12 @@ struct UnitIter {
     u.n_b = min(max(seqlens[u.b], 0), prm.max_blocks_per_seq * kPage);
     return true;
   }
-  // Partial slot of the unit, -1 if its item lies in one part (several divisions: only the epilogue asks)
-  __device__ int slot_of(const Unit& u) const {
+  // Partial slot of the unit, -1 if its item lies in one part (several divisions: only the epilogue asks);
+  // *info = what the combine needs to know about the item
+  __device__ int slot_of(const Unit& u, int2* info) const {
     int p_first, p_last;
     const int nsplit = plan.item_parts(u.it, &p_first, &p_last);
+    *info = make_int2(plan.slot_of(p_first, u.it, p_first), nsplit);
     return nsplit == 1 ? -1 : plan.slot_of(p, u.it, p_first);
   }
 };
@@ -724,7 +726,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
       const int c_first = partner ? 8 : 0;          // first of this warp's eight 32-column chunks
       while (ok && iter.next(u)) {
-        const int slot = partner ? -1 : iter.slot_of(u);
+        int2 info;
+        const int slot = partner ? -1 : iter.slot_of(u, &info);
+        if (tid == 0) prm.item_info[u.it] = info;
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
           const uint32_t s = gt % kNumP, k = gt / kNumP;
           ok = warp_wait<true>(bar(B_PFULL + s), k & 1);

@@ -46,81 +46,117 @@ __global__ void plan_kernel(const int32_t* __restrict__ seqlens, int nrb, int n_
   if (tid == 0) prefix[n_items] = carry;
 }
 
-// One warp per query row.  Items that one part covered entirely were written by the decode kernel
-// and are skipped; items without tiles get out = 0, lse = -inf; split items are merged:
+// One warp per query row.  Items that one part covered entirely were written by the decode kernel and are skipped;
+// items without tiles get out = 0, lse = -inf; split items are merged:
 //   lse = ln sum_s exp(lse_s),  out = sum_s exp(lse_s - lse) * out_s.
-__global__ void combine_kernel(DecodeParams prm) {
+// What the row needs to know about its item (where its partials are) was left in item_info by the decode kernel, so
+// the warp's chain of dependent memory round trips is short: (prefix, item_info) -> (partial lse, partial rows).
+// Up to kFastSplits partials are fetched before any arithmetic.
+constexpr int kFastSplits = 4;
+
+__global__ void __launch_bounds__(128) combine_kernel(DecodeParams prm) {
 #ifdef AMLA_TRACE
   unsigned long long t_ns;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
   if (prm.trace && blockIdx.x == 0 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 0] = t_ns & 0xffffffffull;
 #endif
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-#ifdef AMLA_TRACE
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
-  if (prm.trace && blockIdx.x == 0 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 1] = t_ns & 0xffffffffull;
-  if (prm.trace && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 2] = t_ns & 0xffffffffull;
-#endif   // launched early (programmatic dependent launch): the partials must be complete
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row_global = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   const int rows_padded = prm.nrb * prm.item_rows;
   const int b = row_global / rows_padded;
-  if (b >= prm.B) return;
-  const int rin = row_global - b * rows_padded;   // row within the sequence, padded to row blocks
-  if (rin >= prm.R) return;
+  const int rin = row_global - b * rows_padded;   // row within the sequence, padded to items
+  const bool live = b < prm.B && rin < prm.R;
   const int rb = rin / prm.item_rows, rr = rin % prm.item_rows;   // item of the sequence, row within the item
   const int it = b * prm.nrb + rb;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // launched early (programmatic dependent launch): the partials must be complete
+#ifdef AMLA_TRACE
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
+  if (prm.trace && blockIdx.x == 0 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 1] = t_ns & 0xffffffffull;
+  if (prm.trace && blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 2] = t_ns & 0xffffffffull;
+#endif
+  if (!live) return;
 
-  const Plan plan = Plan::make(prm.prefix, prm.n_items, prm.P, prm.ovh);
-  int p_first, p_last;
-  const int nsplit = plan.L > 0 ? plan.item_parts(it, &p_first, &p_last) : 0;
-  if (nsplit == 1) return;
-
+  const int pa = prm.prefix[it], pe = prm.prefix[it + 1];
+  const int2 info = prm.item_info[it];           // valid only for items with tiles
   __nv_bfloat16* orow = prm.out + (static_cast<size_t>(b) * prm.R + rin) * kDv;
   float* lrow = prm.lse + static_cast<size_t>(b) * prm.R + rin;
-  if (nsplit == 0) {
+  auto write_empty = [&]() {
     for (int c = lane * 8; c < kDv; c += 32 * 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
     if (lane == 0) *lrow = -INFINITY;
-    return;
-  }
-  // lse of the splits: one split per lane (in rounds of 32), so that the loads overlap
-  float mx = -INFINITY;
-  for (int base = 0; base < nsplit; base += 32) {
-    const int sidx = base + lane;
-    if (sidx < nsplit) mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(plan.slot_of(p_first + sidx, it, p_first)) * prm.item_rows + rr]);
-  }
-#pragma unroll
-  for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  if (mx == -INFINITY) {   // no split saw a visible key for this row
-    for (int c = lane * 8; c < kDv; c += 32 * 8) *reinterpret_cast<uint4*>(orow + c) = make_uint4(0, 0, 0, 0);
-    if (lane == 0) *lrow = -INFINITY;
-    return;
-  }
+  };
+  if (pe <= pa) { write_empty(); return; }       // no tiles: no part ever saw this item
+  const int nsplit = info.y;
+  if (nsplit == 1) return;
+
   float acc[16];
+  float tot = 0.f, mx;
+  if (nsplit <= kFastSplits) {
+    // everything is requested before anything is used
+    float ls[kFastSplits];
+    float4 v[kFastSplits][4];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) acc[i] = 0.f;
-  float tot = 0.f;
-  for (int base = 0; base < nsplit; base += 32) {
-    const int sidx = base + lane;
-    int my_slot = 0;
-    float my_w = 0.f;
-    if (sidx < nsplit) {
-      my_slot = plan.slot_of(p_first + sidx, it, p_first);
-      my_w = expf(prm.part_lse[static_cast<size_t>(my_slot) * prm.item_rows + rr] - mx);   // 0 for a split that saw nothing
+    for (int s = 0; s < kFastSplits; ++s) {
+      ls[s] = -INFINITY;
+      if (s < nsplit) {
+        const size_t prow = static_cast<size_t>(Plan::slot_of_split(info.x, s)) * prm.item_rows + rr;
+        ls[s] = prm.part_lse[prow];
+        const float4* src = reinterpret_cast<const float4*>(prm.part_o + prow * kDv);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[s][i] = src[i * 32 + lane];
+      }
     }
-    const int n_here = min(32, nsplit - base);
-#pragma unroll 2
-    for (int j = 0; j < n_here; ++j) {
-      const float w = __shfl_sync(0xffffffffu, my_w, j);
-      const int slot = __shfl_sync(0xffffffffu, my_slot, j);
-      tot += w;
-      const float* src = prm.part_o + (static_cast<size_t>(slot) * prm.item_rows + rr) * kDv;
+    mx = ls[0];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float4 v = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
-        acc[4 * i + 0] += w * v.x; acc[4 * i + 1] += w * v.y;
-        acc[4 * i + 2] += w * v.z; acc[4 * i + 3] += w * v.w;
+    for (int s = 1; s < kFastSplits; ++s) mx = fmaxf(mx, ls[s]);
+    if (mx == -INFINITY) { write_empty(); return; }   // no split saw a visible key for this row
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int s = 0; s < kFastSplits; ++s) {
+      if (s < nsplit) {
+        const float w = expf(ls[s] - mx);             // 0 for a split that saw nothing
+        tot += w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[4 * i + 0] += w * v[s][i].x; acc[4 * i + 1] += w * v[s][i].y;
+          acc[4 * i + 2] += w * v[s][i].z; acc[4 * i + 3] += w * v[s][i].w;
+        }
+      }
+    }
+  } else {
+    // lse of the splits: one split per lane (in rounds of 32), so that the loads overlap
+    mx = -INFINITY;
+    for (int base = 0; base < nsplit; base += 32) {
+      const int sidx = base + lane;
+      if (sidx < nsplit) mx = fmaxf(mx, prm.part_lse[static_cast<size_t>(Plan::slot_of_split(info.x, sidx)) * prm.item_rows + rr]);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (mx == -INFINITY) { write_empty(); return; }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    for (int base = 0; base < nsplit; base += 32) {
+      const int sidx = base + lane;
+      int my_slot = 0;
+      float my_w = 0.f;
+      if (sidx < nsplit) {
+        my_slot = Plan::slot_of_split(info.x, sidx);
+        my_w = expf(prm.part_lse[static_cast<size_t>(my_slot) * prm.item_rows + rr] - mx);
+      }
+      const int n_here = min(32, nsplit - base);
+#pragma unroll 2
+      for (int j = 0; j < n_here; ++j) {
+        const float w = __shfl_sync(0xffffffffu, my_w, j);
+        const int slot = __shfl_sync(0xffffffffu, my_slot, j);
+        tot += w;
+        const float* src = prm.part_o + (static_cast<size_t>(slot) * prm.item_rows + rr) * kDv;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 x = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
+          acc[4 * i + 0] += w * x.x; acc[4 * i + 1] += w * x.y;
+          acc[4 * i + 2] += w * x.z; acc[4 * i + 3] += w * x.w;
+        }
       }
     }
   }
@@ -135,6 +171,10 @@ __global__ void combine_kernel(DecodeParams prm) {
     *reinterpret_cast<uint2*>(orow + i * 128 + lane * 4) = pk;
   }
   if (lane == 0) *lrow = mx + logf(tot);
+#ifdef AMLA_TRACE
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
+  if (prm.trace && lane == 0) atomicMax(prm.trace + 148 * 16 * 128 + 3, t_ns & 0xffffffffull);
+#endif
 }
 
 cudaError_t launch_plan(const DecodeParams& prm, int* prefix_out, cudaStream_t stream) {

@@ -27,10 +27,11 @@ constexpr size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign;
 constexpr int kMaxItems = AMLA_STATIC_MAX_ITEMS;      // (sequence, 128-row block) pairs
 constexpr int kMaxParts = AMLA_STATIC_MAX_SMS / 2;    // clusters
 
-// status | prefix[kMaxItems + 1] | partial lse [2 * parts][128] | partial O [2 * parts][128][512]
+// status | prefix[kMaxItems + 1] | item info [kMaxItems] | partial lse [2 * parts][128] | partial O [2 * parts][128][512]
 constexpr size_t kStatusOff = 0;
 constexpr size_t kPrefixOff = kAlign;
-constexpr size_t kPartLseOff = kPrefixOff + align_up(sizeof(int) * (kMaxItems + 1));
+constexpr size_t kInfoOff = kPrefixOff + align_up(sizeof(int) * (kMaxItems + 1));
+constexpr size_t kPartLseOff = kInfoOff + align_up(sizeof(int2) * kMaxItems);
 constexpr size_t kPartOOff = kPartLseOff + align_up(sizeof(float) * 2 * kMaxParts * amla::kRowBlock);
 constexpr size_t kScratchBytes = kPartOOff + sizeof(float) * 2 * kMaxParts * amla::kRowBlock * amla::kDv;
 static_assert(kScratchBytes <= (40u << 20), "the built-in scratch is meant to stay modest");
@@ -113,6 +114,7 @@ extern "C" int amla_mla_decode_static(const void* q, const void* kv_cache, const
   prm.status = reinterpret_cast<int*>(ws + kStatusOff);
   int* prefix = reinterpret_cast<int*>(ws + kPrefixOff);
   prm.prefix = prefix;
+  prm.item_info = reinterpret_cast<int2*>(ws + kInfoOff);
   prm.part_lse = reinterpret_cast<float*>(ws + kPartLseOff);
   prm.part_o = reinterpret_cast<float*>(ws + kPartOOff);
   prm.scale_log2 = softmax_scale * kLog2e;
