@@ -123,6 +123,28 @@ def time_oracle(w, n_rows):
     return flops / dt / 1e12, dt, R.num_threads(), f"{n_rows} seeded (b,t,h) query rows of the {w.name} workload, all their keys"
 
 
+def config_block(w, nrep=None, eff=None):
+    """The `config` object of the JSON line; the same for both arms (it names the workload, not the arm)."""
+    kv_bytes = w.kv.nbytes
+    if nrep is None:
+        nrep = replica_count(kv_bytes)
+    if eff is None:
+        eff = DEFAULT_FLAGS
+    tot = nrep * kv_bytes / 1e6
+    return {"workload": workload_name(w),
+            "l2": f"{nrep} input replicas rotated between steps ({tot:.0f} MB of KV) " + ("> 126 MB L2" if tot > 126 else "(fits in L2: latency-bound case)"),
+            "rescale": ["alg2", "fold", "fmul"][eff & 3] + f" tau={(eff >> 8) & 15}" + (" unguarded" if eff & 4 else "")}
+
+
+DEFAULT_FLAGS = 0 | (8 << 8)      # AMLA_RESCALE_ALG2 | AMLA_LAZY(8): what amla_mla_decode uses
+
+
+def replica_count(kv_bytes):
+    """Input replicas rotated between steps so that no step finds its KV cache in L2 (126 MB)."""
+    nrep = max(2, int(np.ceil(400e6 / kv_bytes))) if kv_bytes < 400e6 else 2
+    return min(nrep, 8)
+
+
 def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
@@ -141,10 +163,11 @@ def run_reference(args):
     value = float(np.mean(tfl))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(times)), "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(times)), "median_step_ms": 1e3 * float(np.median(times)),
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(w), "sample_rows_per_step": n_rows},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": config_block(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample + " per step"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -159,6 +182,70 @@ def workload_name(w):
 
 
 # --------------------------------------------------------------------------------------------------
+def roofline_of(w, dec_ms, peaks, peak_kind):
+    """Roofline object for the decode kernel of one workload: the slower of (FLOPs at the measured bf16 peak) and
+    (algorithmic bytes at the measured HBM peak) is the bound; achieved = that quantity / the kernel's duration."""
+    flops, alg_bytes = w.flops(), w.algorithmic_bytes()
+    hbm_peak, tc_peak = float(peaks["hbm_gbs"]), float(peaks["bf16_tflops"])
+    if alg_bytes / (hbm_peak * 1e9) >= flops / (tc_peak * 1e12):
+        ach = alg_bytes / (dec_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak}
+    else:
+        ach = flops / (dec_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
+    roof.update({"traffic": None, "peak_kind": f"of {peak_kind} (burst)", "kernel_ms": dec_ms,
+                 "kernel_tflops": flops / (dec_ms * 1e-3) / 1e12,
+                 "frac_of_bf16_measured": flops / (dec_ms * 1e-3) / 1e12 / tc_peak,
+                 "frac_of_bf16_nominal_2250": flops / (dec_ms * 1e-3) / 1e12 / 2250.0,
+                 "kernel_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9, "algorithmic_bytes": alg_bytes, "flops": flops})
+    return roof
+
+
+class DeviceRun:
+    """One workload resident on the device (rotating input replicas) and the timing of its decode calls."""
+
+    def __init__(self, w, dev, local, flags):
+        import torch
+        from paper_2509_25224_b200 import binding
+        self.torch, self.binding, self.w, self.flags = torch, binding, w, flags
+        self.nrep = replica_count(w.kv.nbytes)
+        self.reps = []
+        for _ in range(self.nrep):
+            self.reps.append((torch.from_numpy(w.q.view(np.int16)).to(dev).view(torch.bfloat16),
+                              torch.from_numpy(w.kv.view(np.int16)).to(dev).view(torch.bfloat16),
+                              torch.from_numpy(w.block_table).to(dev), torch.from_numpy(w.seqlens).to(dev)))
+        self.out = torch.empty((w.B, w.Sq, w.H, 512), dtype=torch.bfloat16, device=dev)
+        self.lse = torch.empty((w.B, w.Sq, w.H), dtype=torch.float32, device=dev)
+        self.ws = torch.empty(binding.workspace_size(w.B, w.Sq, w.H, w.max_blocks_per_seq, local), dtype=torch.uint8, device=dev)
+
+    def step(self, i, flags="same"):
+        q, kv, bt, sl = self.reps[i % self.nrep]
+        self.binding.mla_decode(q, kv, bt, sl, self.w.scale, self.out, self.lse, self.ws, self.flags if flags == "same" else flags)
+
+    def timed(self, steps, barrier, flags="same"):
+        """(total ms, per-step ms list) of `steps` calls bracketed by barrier + synchronize, CUDA events per step."""
+        torch = self.torch
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        evs[0].record()
+        for i in range(steps):
+            self.step(i, flags)
+            evs[i + 1].record()
+        barrier()
+        return evs[0].elapsed_time(evs[-1]), [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+
+    def kernel_times(self, steps, flags="same"):
+        """Mean (schedule, decode, combine) ms from events the library records around its launches."""
+        self.binding.profile_enable(True)
+        ks = []
+        for i in range(steps):
+            self.step(i, flags)
+            ks.append(self.binding.profile_last_ms())
+        self.binding.profile_enable(False)
+        self.torch.cuda.synchronize()
+        return tuple(float(np.mean([k[j] for k in ks])) for j in range(3))
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -173,28 +260,11 @@ def run_gpu(args):
 
     w = synth.CONFIGS[args.config]()
     B, Sq, H = w.B, w.Sq, w.H
-    # input replicas rotated between steps so that no step finds its KV cache in L2 (126 MB)
-    kv_bytes = w.kv.nbytes
-    nrep = max(2, int(np.ceil(400e6 / kv_bytes))) if kv_bytes < 400e6 else 2
-    nrep = min(nrep, 8)
-    reps = []
-    for _ in range(nrep):
-        q = torch.from_numpy(w.q.view(np.int16)).to(dev).view(torch.bfloat16)
-        kv = torch.from_numpy(w.kv.view(np.int16)).to(dev).view(torch.bfloat16)
-        bt = torch.from_numpy(w.block_table).to(dev)
-        sl = torch.from_numpy(w.seqlens).to(dev)
-        reps.append((q, kv, bt, sl))
-    out = torch.empty((B, Sq, H, 512), dtype=torch.bfloat16, device=dev)
-    lse = torch.empty((B, Sq, H), dtype=torch.float32, device=dev)
-    ws = torch.empty(binding.workspace_size(B, Sq, H, w.max_blocks_per_seq, local), dtype=torch.uint8, device=dev)
-    flags = None if args.mode is None and args.tau is None else (
+    flags = None if args.mode is None and args.tau is None and not args.rows128 else (
         {"alg2": 0, "fold": 1, "fmul": 2}[args.mode or "alg2"] | binding.lazy(binding.DEFAULT_TAU if args.tau is None else args.tau)
-        | (binding.FLAG_UNGUARDED_ADD if args.unguarded else 0))
+        | (binding.FLAG_UNGUARDED_ADD if args.unguarded else 0) | (binding.FLAG_KERNEL_ROWS128 if args.rows128 else 0))
     eff = binding.DEFAULT_FLAGS if flags is None else flags
-
-    def step(i):
-        q, kv, bt, sl = reps[i % nrep]
-        binding.mla_decode(q, kv, bt, sl, w.scale, out, lse, ws, flags)
+    run = DeviceRun(w, dev, local, flags)
 
     def barrier():
         if world > 1:
@@ -202,35 +272,20 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     for i in range(max(args.warmup, 3)):
-        step(i)
-    binding.check_status(ws)
+        run.step(i)
+    binding.check_status(run.ws)
 
     # ---- timed region: K steps, device-resident inputs
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    barrier()
-    evs[0].record()
-    for i in range(args.steps):
-        step(i)
-        evs[i + 1].record()
-    barrier()
+    total_ms, per_step = run.timed(args.steps, barrier)
     launches = binding.last_launch_count() * args.steps
-    total_ms = evs[0].elapsed_time(evs[-1])
-    per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
-
     # ---- same K steps again with per-kernel events (decode kernel duration for the roofline)
-    binding.profile_enable(True)
-    kern_ms = []
-    for i in range(args.steps):
-        step(i)
-        kern_ms.append(binding.profile_last_ms())
-    binding.profile_enable(False)
-    torch.cuda.synchronize()
+    plan_ms, dec_ms, comb_ms = run.kernel_times(args.steps)
     clocks = sampler.stop() if rank == 0 else None
-    binding.check_status(ws)
+    binding.check_status(run.ws)
 
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -255,53 +310,67 @@ def run_gpu(args):
     if world > 1:
         dist.all_reduce(t2, op=dist.ReduceOp.MAX)
     e2e_value = world * flops * e2e_steps / (float(t2.item()) * 1e-3) / 1e12
+    h2d, d2h = sess.h2d_bytes, sess.d2h_bytes
+    del sess
+
+    # ---- the other configurations, on rank 0 at N = 1 (roofline fraction for every configuration)
+    per_config = {}
+    if rank == 0 and world == 1 and not args.no_per_config:
+        traffic = load_traffic()
+        ksteps = max(10, min(args.steps, 100))
+
+        def entry(r, wk, fl="same"):
+            for i in range(5):
+                r.step(i, fl)
+            tot, per = r.timed(ksteps, barrier, fl)
+            _, dms, cms = r.kernel_times(min(ksteps, 50), fl)
+            rf = roofline_of(wk, dms, peaks, peak_kind)
+            return {"ms_per_step": tot / ksteps, "median_step_ms": statistics.median(per), "tflops": wk.flops() * ksteps / (tot * 1e-3) / 1e12,
+                    "kernel_ms": dms, "combine_ms": cms, "kernel_tflops": rf["kernel_tflops"], "bound": rf["bound"],
+                    "frac": rf["frac"], "frac_of_bf16_measured": rf["frac_of_bf16_measured"], "steps": ksteps,
+                    "traffic": traffic.get(wk.name), "workload": workload_name(wk)}
+
+        per_config[w.name] = {"ms_per_step": total_ms / args.steps, "median_step_ms": statistics.median(per_step),
+                              "tflops": flops * args.steps / (total_ms * 1e-3) / 1e12, "kernel_ms": dec_ms, "combine_ms": comb_ms,
+                              **{k: v for k, v in roofline_of(w, dec_ms, peaks, peak_kind).items() if k in ("kernel_tflops", "bound", "frac", "frac_of_bf16_measured")},
+                              "steps": args.steps, "traffic": traffic.get(w.name), "workload": workload_name(w)}
+        tau0 = binding.RESCALE_ALG2 | binding.lazy(0)
+        if w.name in ("dsv3", "long") and flags is None:
+            per_config[w.name + " tau=0"] = entry(run, w, tau0)
+        del run
+        torch.cuda.empty_cache()
+        for name in synth.CONFIGS:
+            if name == w.name:
+                continue
+            wk = synth.CONFIGS[name]()
+            r = DeviceRun(wk, dev, local, None)
+            per_config[name] = entry(r, wk)
+            if name in ("dsv3", "long"):
+                per_config[name + " tau=0"] = entry(r, wk, tau0)
+            binding.check_status(r.ws)
+            del r
+            torch.cuda.empty_cache()
 
     if rank == 0:
-        dec_ms = float(np.mean([k[1] for k in kern_ms]))
-        plan_ms = float(np.mean([k[0] for k in kern_ms]))
-        comb_ms = float(np.mean([k[2] for k in kern_ms]))
-        alg_bytes = w.algorithmic_bytes()
-        hbm_peak = float(peaks["hbm_gbs"])
-        tc_peak = float(peaks["bf16_tflops"])
-        t_bytes = alg_bytes / (hbm_peak * 1e9)
-        t_flops = flops / (tc_peak * 1e12)
-        if t_bytes >= t_flops:
-            ach = alg_bytes / (dec_ms * 1e-3) / 1e9
-            roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak}
-        else:
-            ach = flops / (dec_ms * 1e-3) / 1e12
-            roof = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak}
-        roof.update({
-            "traffic": None, "peak_kind": f"of {peak_kind} (burst)", "kernel": "decode_tc_kernel",
-            "kernel_ms": dec_ms, "schedule_ms": plan_ms, "combine_ms": comb_ms,
-            "kernel_tflops": flops / (dec_ms * 1e-3) / 1e12,
-            "frac_of_bf16_measured": flops / (dec_ms * 1e-3) / 1e12 / tc_peak,
-            "frac_of_bf16_nominal_2250": flops / (dec_ms * 1e-3) / 1e12 / 2250.0,
-            "kernel_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9,
-            "algorithmic_bytes": alg_bytes, "flops": flops,
-        })
-        # DRAM bytes per launch from the committed ncu capture; only valid for the kernel sources it was taken with
-        traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(traffic_file):
-            with open(traffic_file) as f:
-                tr = json.load(f)
-            if tr.get("source_sha256") == kernel_source_hash():
-                roof["traffic"] = tr.get(w.name)
+        roof = roofline_of(w, dec_ms, peaks, peak_kind)
+        roof.update({"kernel": "decode_quad_kernel" if (Sq * H > 128 and not args.rows128) else "decode_tc_kernel",
+                     "schedule_ms": plan_ms, "combine_ms": comb_ms})
+        roof["traffic"] = load_traffic().get(w.name)
         n_rows = {"tiny": 16, "dsv3": 4096, "mtp": 2048, "stress": 1024, "long": 256}[w.name]
         tf, dt, cores, sample = time_oracle(w, n_rows)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms_max / args.steps, "median_step_ms": statistics.median(per_step),
+            "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_name(w), "l2": f"{nrep} input replicas rotated between steps "
-                       f"({nrep * kv_bytes / 1e6:.0f} MB of KV) > 126 MB L2", "rescale": ["alg2", "fold", "fmul"][eff & 3] + f" tau={(eff >> 8) & 15}" + (" unguarded" if eff & 4 else ""),
-                       "median_step_ms": statistics.median(per_step)},
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": sess.h2d_bytes, "d2h_bytes_per_step": sess.d2h_bytes,
+            "config": config_block(w, None, eff),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": launches,
             "clocks": clocks,
             "roofline": roof,
             "cpu_baseline": {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": dt},
+            "per_config": per_config,
         }
         print(json.dumps(line))
     if world > 1:
@@ -309,16 +378,29 @@ def run_gpu(args):
     return 0
 
 
+def load_traffic():
+    """DRAM bytes per launch from the committed ncu captures; only valid for the kernel sources they were taken with."""
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        with open(traffic_file) as f:
+            tr = json.load(f)
+        if tr.get("source_sha256") == kernel_source_hash():
+            return {k: v for k, v in tr.items() if k != "source_sha256"}
+    return {}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="dsv3", choices=list(synth.CONFIGS))
     ap.add_argument("--mode", default=None, choices=["alg2", "fold", "fmul"], help="rescale variant (default: the library's)")
     ap.add_argument("--tau", type=int, default=None, help="lazy-reference threshold in octaves, 0..15 (default: the library's)")
     ap.add_argument("--unguarded", action="store_true", help="literal single integer add (measurement only)")
+    ap.add_argument("--rows128", action="store_true", help="A/B: independent 128-row blocks instead of the 256-row kernel (measurement only)")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other configurations")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
