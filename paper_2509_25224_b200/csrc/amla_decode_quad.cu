@@ -6,8 +6,8 @@
 //       part in shared memory) and loads ONE page of every tile: S = Q K^T is a pair MMA (M = 256, N = 128, K = 16,
 //       issued by rank 0) whose B operand is split over the two CTAs, so that every key row enters the shared
 //       memory of one SM only and serves all 256 query rows.  Each CTA runs the softmax of its own 128 rows
-//       (Algorithm 2's per-row recurrence, lines 5-12) and ships P~ = bf16(P * S16) and the per-row integers N to
-//       "its" value CTA.
+//       (Algorithm 2's per-row recurrence, lines 5-12; two threads per row, one per page of the tile) and ships
+//       P~ = bf16(P * S16) and the per-row integers N to "its" value CTA by asynchronous remote stores.
 //   value pair (cluster ranks 2, 3)   CTA j holds the FP32 accumulator O of rows 128 j .. in its tensor memory; the
 //       P~ V product is a pair MMA (M = 256, N = 256) whose B operand (V: 128 of the 256 columns per CTA) is again
 //       split, so each value CTA loads half of every V tile.  The correction warps apply N to the bit patterns of O
@@ -31,8 +31,7 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kNumCopyWarps = 4;
-constexpr int kThreads = 32 * (6 + kNumCopyWarps);   // warps 0-3: softmax / correction, 4: TMA producers, 5: MMA issuer + TMEM alloc, 6-9: P copy / correction partners
+constexpr int kThreads = 32 * 10;   // warps 0-3 and 6-9: softmax (score CTAs) / correction + epilogue (value CTAs), 4: TMA producers, 5: MMA issuer or relay, TMEM alloc
 constexpr int kTileKeys = 2 * kPage;                 // keys per schedule tile
 constexpr int kItemRows = 2 * kRowBlock;             // query rows per work item
 constexpr uint32_t kBoxBytes = 64 * 64 * 2;          // one 64-key x 64-column TMA box
@@ -49,8 +48,9 @@ constexpr int kNumKSlots = 6;                        // two tiles in flight per 
 constexpr uint32_t kKSlotBytes = 3 * kBoxBytes;      // 64 keys x 192 columns: [8 row groups][3 blocks][8 rows][128 B]
 constexpr uint32_t kKGroupStride = 3 * 1024;
 constexpr uint32_t kOffQRope = 0;                    // 128 rows x 64 bf16, 128-byte swizzle
-constexpr uint32_t kOffStage = 128 * 64 * 2;         // one staged page (P~, N, final scalars)
-constexpr uint32_t kOffK = kOffStage + kPStride;
+constexpr uint32_t kOffXchg = 128 * 64 * 2;          // float [2 exchanges in flight][2 warpgroups][128 rows]: what the two threads of a row tell each other
+constexpr uint32_t kOffStage = kOffXchg + 2 * 1024;  // 8 softmax warps x 4 KB: a warp's 32 rows of P~, in the byte order of the P buffer
+constexpr uint32_t kOffK = kOffStage + 8 * 4096;
 constexpr uint32_t kEndA = kOffK + kNumKSlots * kKSlotBytes;
 // ---- value CTA
 constexpr int kNumVSlots = 4;
@@ -85,7 +85,7 @@ constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
 #define QSTAMP_NS(smem_base_, idx) do { } while (0)
 #endif
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
-static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0 && kOffStage % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kQCol = 0;            // score CTA: latent part of Q, 256 columns (two bf16 per column)
@@ -99,7 +99,7 @@ constexpr uint16_t kMaskScore = 0x3, kMaskValue = 0xC, kMaskAll = 0xF;
 // and in the odd CTA the otherwise idle warp 5 relays each completed phase as ONE arrival on the even CTA's copy.
 enum { X_PV = 0, X_COMMON = X_PV + kNumP };
 enum { A_KFULL = X_COMMON /* even CTA */, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2 /*R*/,
-       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2 /*R*/, A_QFREE, A_NUM };
+       A_XCHG = A_SEMPTY + 2, A_QREADY = A_XCHG + 4 /*R*/, A_QFREE, A_NUM };
 enum { B_VFULL = X_COMMON /* even CTA */, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP /*R*/,
        B_NUM = B_OREADY + kNumP };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
@@ -202,20 +202,30 @@ __device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int
 
 struct RoleCtx {
   uint32_t smem_base, bars, tbase;
+  uint32_t peer_base, peer_bars;                // this score CTA's value CTA (cluster addresses)
   int half, tid;                                // half: which 128 rows of the 256-row block this CTA owns
   int part;
 };
 
-// The softmax warpgroup's work on one unit: its 128-key score tiles; the final scalars travel with the last page.
-// Returns (pages so far) << 32 | (score tiles so far) << 1 | ok.
+// One softmax warp's work on one unit.  Two threads share a query row: the thread of warpgroup A (warps 0-3) takes
+// the first 64-key page of every 128-key score tile, the thread of warpgroup B (warps 6-9, which reach the same
+// tensor-memory lanes as warps 2, 3, 0, 1) the second.  Each reads its 64 scores into registers (the score tile is
+// free for the next QK^T from then on), the two exchange their maxima through shared memory and run Algorithm 2's
+// per-row recurrence (lines 5-12) on the same inputs, so both hold the same state; the row sum of line 6 is kept as
+// two partial sums that meet at the end of the unit.  P~ = bf16(P * S16) and the row's integer N (first page only:
+// the second page leaves O alone) go straight into a P buffer of this CTA's value CTA by asynchronous remote stores
+// counted on its barrier; with the unit's last page travel the final scalars 1/(l*S16) and lse (line 20).
+// Returns (score tiles so far) << 1 | ok.
 template <int kMode>
-__device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const RoleCtx c, const Unit u, uint32_t gt, uint32_t gs) {
+__device__ __noinline__ uint32_t softmax_unit(const DecodeParams prm, const RoleCtx c, const Unit u, uint32_t gs, uint32_t un) {
   const int tid = c.tid, wid = tid >> 5, lane = tid & 31;
   const uint32_t smem_base = c.smem_base, bars = c.bars, tbase = c.tbase;
   auto bar = [&](int i) { return bars + 8u * i; };
   bool ok = true;
-  const int r = tid;
-  const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
+  const int hsel = wid >= 6 ? 1 : 0;                   // which page of every tile
+  const int quarter = wid & 3;                         // tensor-memory lane quarter of this warp
+  const int r = quarter * 32 + lane;                   // query row within this CTA's 128
+  const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
   const bool scale_nonneg = prm.scale_log2 >= 0.f;
   const uint32_t mask_fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
   RowState st;
@@ -223,6 +233,17 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
   const int tok = (u.r0 + c.half * kRowBlock + r) / prm.H;
   const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);               // keys 0..visible-1 are seen by this row
   const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kTileKeys;   // tiles from here on may hold hidden keys
+  uint32_t xc = gs + un;                                // exchanges so far: one per tile, one at the end of a unit
+  const uint32_t xbar = bar(A_XCHG + quarter);
+  // tells the row's other thread `mine`, returns what it told
+  auto exchange = [&](float mine) -> float {
+    const uint32_t slot = smem_base + kOffXchg + (xc & 1) * 1024;
+    st_shared_b32(slot + (hsel * 128 + r) * 4, __float_as_uint(mine));
+    warp_arrive(xbar, lane);
+    ok = warp_wait(xbar, xc & 1);
+    ++xc;
+    return __uint_as_float(ld_shared_b32(slot + ((hsel ^ 1) * 128 + r) * 4));
+  };
 
   for (int t = u.t0; t < u.t1 && ok; ++t, ++gs) {
     const uint32_t sb = gs & 1;
@@ -231,14 +252,20 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
     tc_fence_after_sync();
     if (tid == 0) QSTAMP(c.smem_base, 2, gs);
     if (tid == 0 && gs == 0) QSTAMP_NS(c.smem_base, 6);
-    const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
-    const int nvis = visible - t * kTileKeys;            // keys of this tile the row sees (may be <= 0)
+    const uint32_t scol = tbase + lane_base + kSCol + 128 * sb + 64 * hsel;
+    const int nvis = visible - t * kTileKeys - 64 * hsel;    // keys of this page the row sees (may be <= 0)
     const bool last_tile = t + 1 == u.t1;
+    uint32_t b0[32], b1[32];
+    tmem_ld_32x32b_x32(scol, b0);
+    tmem_ld_32x32b_x32(scol + 32, b1);
+    tmem_wait_ld();
+    tc_fence_before_sync();
+    warp_arrive(bar(A_SEMPTY + sb), lane);                   // the scores are in registers
+    if (tid == 0) QSTAMP(c.smem_base, 3, gs);
     auto tile_body = [&](auto general_c) {
       constexpr bool kGeneral = decltype(general_c)::value;
       constexpr bool masked = kGeneral;
       const bool scale_nn = kGeneral ? scale_nonneg : true;
-      uint32_t b0[32], b1[32];
       // lines 5-6: running max on the raw scores (the scale is folded into the FMA below)
       float ext = scale_nn ? -INFINITY : INFINITY, ext_b = ext;
       auto chunk_max = [&](uint32_t (&v)[32], int col0) {
@@ -260,18 +287,12 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           }
         }
       };
-      tmem_ld_32x32b_x32(scol, b0);
-#pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
-        tmem_wait_ld();
-        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
-        chunk_max(b0, 64 * h);
-        tmem_wait_ld();
-        tmem_ld_32x32b_x32(scol + (h == 0 ? 64 : 0), b0);   // second page, or the first chunk again for the second pass
-        chunk_max(b1, 64 * h + 32);
-      }
+      chunk_max(b0, 0);
+      chunk_max(b1, 32);
       ext = scale_nn ? fmaxf(ext, ext_b) : fminf(ext, ext_b);
-      const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
+      const float mine = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
+      const float tmax = fmaxf(mine, exchange(mine));
+      if (!ok) return;
       const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
       if (tid == 0) QSTAMP(c.smem_base, 13, gs);
       // Line 10's factor S16 goes into the exponential's argument (the remark after Algorithm 2).  The row sum of
@@ -304,56 +325,58 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           }
         }
       };
-#pragma unroll 1
-      for (int h = 0; h < 2; ++h) {
-        tmem_wait_ld();
-        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
-        chunk_exp(b0, 64 * h, 0);
-        tmem_wait_ld();
-        if (h == 0) {
-          tmem_ld_32x32b_x32(scol + 64, b0);
-        } else {                       // the score tile has been read for the last time
-          tc_fence_before_sync();
-          warp_arrive(bar(A_SEMPTY + sb), lane);
-          if (tid == 0) QSTAMP(c.smem_base, 3, gs);
-        }
-        // One staging buffer: the copy warps of the previous page must have read it into registers.  The barrier
-        // is probed ahead of the last chunk's arithmetic, so that the probe's latency is not exposed.
-        const bool stage_free = gt == 0 || mbar_probe(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
-        chunk_exp(b1, 64 * h + 32, 16);
-        const uint32_t s2 = gt & 1;
-        if (!__all_sync(0xffffffffu, stage_free)) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
-        if (!ok) break;
-        if (tid == 0) QSTAMP(c.smem_base, 14, gt);
-        const uint32_t stg = smem_base + kOffStage;
+      chunk_exp(b0, 0, 0);
+      chunk_exp(b1, 32, 16);
+      {
+        float s0, s1;
+        unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
+        st.l = st.l * sp.l_up + __fdividef((rs0 + s0) + (rs1 + s1), sp.p_scale);   // this thread's share of the row sum
+      }
+      // ---- ship the page: P~ (128 B of this row), the row's word N, and with the unit's last page the final scalars
+      const uint32_t stage = smem_base + kOffStage + (hsel * 4 + quarter) * 4096;
 #pragma unroll
-        for (int cc = 0; cc < 8; ++cc)
-          st_shared_v4(stg + sw128_offset(r, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-        // the rescale (if any) belongs to the first page; the second leaves O alone
-        const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
-                                            : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
-        st_shared_b32(stg + kNOff + r * 4, nword);
-        if (h == 1) {
-          float s0, s1;
-          unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
-          st.l = st.l * sp.l_up + __fdividef((rs0 + s0) + (rs1 + s1), sp.p_scale);
-          if (last_tile) {
-            // line 20 scalars: 1 / (l * S16) and lse = m + ln l; they ride with the unit's last page
-            const bool live = st.l > 0.f;
-            const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
-            const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
-            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(stg + kFinOff + r * 8), "r"(__float_as_uint(inv)), "r"(__float_as_uint(lse)) : "memory");
-          }
+      for (int cc = 0; cc < 8; ++cc)
+        st_shared_v4(stage + sw128_offset(lane, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+      __syncwarp();
+      const uint32_t gp = 2 * gs + hsel;                     // page number within the cluster's work
+      const uint32_t pb = gp % kNumP;
+      ok = warp_wait(bar(X_PV + pb), ((gp / kNumP) & 1) ^ 1);     // the P V that last read the buffer is done
+      if (!ok) return;
+      const bool with_fin = last_tile && hsel == 1;
+      const uint32_t pfull = c.peer_bars + 8u * (B_PFULL + pb);
+      const uint32_t dstp = c.peer_base + kOffP + pb * kPStride;
+      if (quarter == 0 && lane == 0) { QSTAMP(c.smem_base, 5, gp); mbar_arrive_expect_tx_cluster(pfull, with_fin ? kPXferLast : kPXfer); }
+      // A thread's 128 bytes are eight 16-byte pieces of one row; sent as they are, every store instruction of the
+      // warp would be 32 separate small remote writes (measured: ~290 clk per instruction).  The warp's 32 rows are a
+      // contiguous 4 KB block of the P buffer, so it goes through a 4 KB staging block of the warp's own and leaves
+      // in instructions that cover 512 contiguous bytes each.
+      uint32_t v[8][4];
+#pragma unroll
+      for (int cc = 0; cc < 8; ++cc)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[cc][0]), "=r"(v[cc][1]), "=r"(v[cc][2]), "=r"(v[cc][3])
+                     : "r"(stage + cc * 512 + lane * 16));
+#pragma unroll
+      for (int cc = 0; cc < 8; ++cc)
+        st_async_v4(dstp + quarter * 4096 + cc * 512 + lane * 16, v[cc][0], v[cc][1], v[cc][2], v[cc][3], pfull);
+      const uint32_t nword = (kMode == 2) ? __float_as_uint(hsel == 0 ? sp.l_up : 1.f)
+                                          : static_cast<uint32_t>(hsel == 0 ? sp.n_bits : 0);
+      st_async_b32(dstp + kNOff + r * 4, nword, pfull);
+      if (tid == 0) QSTAMP(c.smem_base, 4, gp);
+      if (last_tile) {
+        // line 20 scalars: 1 / (l * S16) and lse = m + ln l, from both threads' shares of the row sum
+        const float l_all = st.l + exchange(st.l);
+        if (ok && hsel == 1) {
+          const bool live = l_all > 0.f;
+          const float inv = live ? 1.f / (l_all * st.s_out) : 0.f;
+          const float lse = live ? (st.m2 + log2f(l_all)) * kLn2 : -INFINITY;
+          st_async_v2(dstp + kFinOff + r * 8, __float_as_uint(inv), __float_as_uint(lse), pfull);
         }
-        mbar_arrive(bar(A_PSTAGED + s2));
-        if (tid == 0) QSTAMP(c.smem_base, 4, gt);
-        ++gt;
       }
     };
     if (t >= first_masked_tile || !scale_nonneg) tile_body(std::true_type{});
     else tile_body(std::false_type{});
   }
-  return (static_cast<uint64_t>(gt) << 32) | (static_cast<uint64_t>(gs) << 1) | (ok ? 1u : 0u);
+  return (gs << 1) | (ok ? 1u : 0u);
 }
 
 // Relay warp of a pair's odd CTA: lane l < n_lanes watches barrier `first + l` of this CTA and passes each of its
@@ -415,9 +438,9 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     if (is_score) {
       for (int i = 0; i < kNumKSlots; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
       for (int i = 0; i < 2; ++i) {
-        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), leader ? 5 : 4);   // 4 softmax warps (+ the odd CTA's relay)
-        mbar_init(bar(A_PSTAGED + i), 128); mbar_init(bar(A_STAGEFREE + i), 2);
+        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), leader ? 9 : 8);   // 8 softmax warps (+ the odd CTA's relay)
       }
+      for (int i = 0; i < 4; ++i) mbar_init(bar(A_XCHG + i), 2);                        // the two warps that share 32 rows
       mbar_init(bar(A_QREADY), leader ? 9 : 8);                                         // 8 loading warps (+ relay)
       mbar_init(bar(A_QFREE), 1);
     } else {
@@ -490,33 +513,47 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
   if (is_score) {
     // ======================================================================= score CTAs
     uint32_t gs = 0;    // score tiles so far
-    if (wid < 4) {
-      // ---- softmax warpgroup: thread = query row
-      const int r = tid;
-      const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
-      const RoleCtx ctx{smem_base, bars, tbase, half, tid, part};
+    if (wid < 4 || wid >= 6) {
+      // ---- softmax warps: A = warps 0-3 (first page of every tile), B = warps 6-9 (second page).  At the start of
+      // a unit they bring in its Q rows: A the first 256 latent columns, B the other 256 and the RoPE columns.
+      const bool grp_b = wid >= 6;
+      const int qr = (wid & 3) * 32 + lane;
+      const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+      const RoleCtx ctx{smem_base, bars, tbase, myV_base, myV_bars, half, tid, part};
       while (ok && iter.next(u)) {
         ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);      // the previous unit's QK^T is finished with Q
         if (!ok) break;
         tc_fence_after_sync();
         if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 8 + 4 * un); };
         {
-          const int row = u.r0 + half * kRowBlock + r;
+          const int row = u.r0 + half * kRowBlock + qr;
           const bool valid = row < prm.R;
           const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDqk);
-          load_q_latent(qrow, valid, 0, tbase + lane_base + kQCol);
+          load_q_latent(qrow, valid, grp_b ? 4 : 0, tbase + q_lane_base + kQCol);
+          if (grp_b) {
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+              const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
+              st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
+            }
+          }
           tmem_wait_st();
+          if (grp_b) fence_proxy_async_smem();
         }
         tc_fence_before_sync();
         warp_arrive(bar(A_QREADY), lane);
         if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 9 + 4 * un); };
-        const uint64_t ret = softmax_unit<kMode>(prm, ctx, u, gt, gs);
-        gt = static_cast<uint32_t>(ret >> 32);
-        gs = static_cast<uint32_t>(ret & 0xffffffffu) >> 1;
+        if (grp_b) {                               // the next unit's Q goes to L2 while this one is computed
+          UnitIter peek = iter;
+          Unit nu;
+          if (peek.next(nu)) prefetch_q_row(prm, nu, half * kRowBlock + qr);
+        }
+        const uint32_t ret = softmax_unit<kMode>(prm, ctx, u, gs, un);
+        gs = ret >> 1;
         ok = (ret & 1u) != 0;
         ++un;
       }
-      if (!ok) report_timeout(prm.status);
+      if (!ok && lane == 0) report_timeout(prm.status);
     } else if (wid == 4) {
       // ---- TMA producers: K.  This CTA loads page (2 t + half) of every tile t, three slots of 192 columns; lane l
       // owns ring slot l and polls without blocking.  The bytes of both CTAs' halves are counted on the even CTA's
@@ -629,73 +666,13 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       } else if (!leader) {
         // ---- relay (odd CTA): lanes 0, 1 pass on the completed phases of SEMPTY[lane] (the tiles with that buffer),
         // lane 2 those of QREADY (one per unit)
-        static_assert(A_QREADY == A_SEMPTY + 2 + 2 + 2, "lane 2 is moved onto QREADY below");
+
         int n_units = 0, n_tiles = 0;
         while (iter.next(u)) { ++n_units; n_tiles += u.t1 - u.t0; }
         const int phases = lane == 2 ? n_units : lane < 2 ? (n_tiles + 1 - lane) / 2 : 0;
-        const int first = lane == 2 ? A_QREADY - 2 : A_SEMPTY;
+        const int first = lane == 2 ? A_QREADY - 2 : A_SEMPTY;     // lane 2 lands on QREADY
         if (!relay_phases<false>(bars, lead_bars, first, lane, phases) && lane == 0) report_timeout(prm.status);
       }
-    } else if (wid >= 6 && wid < 6 + kNumCopyWarps) {
-      // ---- copy warps: staged P~ / N (and, with a unit's last page, the final scalars) -> a free P buffer of this
-      // CTA's value CTA, by asynchronous remote stores counted on its PFULL barrier.  Warps c and c + 2 serve the
-      // pages of parity c and move one half of the buffer each.
-      const uint32_t c = (wid - 6) & 1, hv = (wid - 6) >> 1;
-      constexpr int kChunks = 18;                         // 512-byte chunks per warp (33 or 35 in total)
-      const int qr = (wid & 3) * 32 + lane;
-      const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
-      while (ok && iter.next(u)) {
-        {
-          ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const int row = u.r0 + half * kRowBlock + qr;
-          const bool valid = row < prm.R;
-          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDqk);
-          load_q_latent(qrow, valid, 4, tbase + q_lane_base + kQCol);
-#pragma unroll
-          for (int cc = 0; cc < 8; ++cc) {
-            const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
-            st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
-          }
-          tmem_wait_st();
-          fence_proxy_async_smem();
-          tc_fence_before_sync();
-          warp_arrive(bar(A_QREADY), lane);
-          ++un;
-          UnitIter peek = iter;
-          Unit nu;
-          if (peek.next(nu)) prefetch_q_row(prm, nu, half * kRowBlock + qr);
-        }
-        const int npages = 2 * (u.t1 - u.t0);
-        for (int pi = 0; pi < npages; ++pi, ++gt) {
-          if ((gt & 1) != c) continue;
-          const bool last = pi + 1 == npages;
-          const int nchunks = last ? 35 : 33;
-          const uint32_t pb = gt % kNumP;
-          ok = warp_wait(bar(A_PSTAGED + c), (gt >> 1) & 1);
-          if (!ok) break;
-          const uint32_t src = smem_base + kOffStage + (hv * kChunks * 32 + lane) * 16;
-          uint32_t v[kChunks][4];
-#pragma unroll
-          for (int i = 0; i < kChunks; ++i) {
-            if (static_cast<int>(hv) * kChunks + i < nchunks)
-              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i][0]), "=r"(v[i][1]), "=r"(v[i][2]), "=r"(v[i][3]) : "r"(src + i * 512));
-          }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(A_STAGEFREE + c));
-          ok = warp_wait(bar(X_PV + pb), ((gt / kNumP) & 1) ^ 1);      // the P V that last read the buffer is done
-          if (!ok) break;
-          const uint32_t pfull = myV_bars + 8u * (B_PFULL + pb);
-          const uint32_t dstp = myV_base + kOffP + pb * kPStride + (hv * kChunks * 32 + lane) * 16;
-          if (lane == 0 && hv == 0) { QSTAMP(smem_base, 5, gt); mbar_arrive_expect_tx_cluster(pfull, last ? kPXferLast : kPXfer); }
-#pragma unroll
-          for (int i = 0; i < kChunks; ++i) {
-            if (static_cast<int>(hv) * kChunks + i < nchunks) st_async_v4(dstp + i * 512, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
-          }
-        }
-      }
-      if (!ok && lane == 0) report_timeout(prm.status);
     }
   } else {
     // ======================================================================= value CTAs
