@@ -58,8 +58,7 @@ constexpr uint32_t kVHalfBytes = 2 * kBoxBytes;      // 64 keys x 128 columns: [
 constexpr uint32_t kVSlotBytes = 2 * kVHalfBytes;    // one page: this CTA's 128 columns of either 256-column half of V
 constexpr uint32_t kOffV = 0;
 constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;
-constexpr uint32_t kOffEpi = kOffP + kNumP * kPStride;
-constexpr uint32_t kEndB = kOffEpi + 4 * 32 * 128;
+constexpr uint32_t kEndB = kOffP + kNumP * kPStride;
 // ---- all four: barriers at the same offset, so that one multicast commit reaches them
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
 constexpr uint32_t kBarBytes = 512;
@@ -678,7 +677,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     // ======================================================================= value CTAs
     if (wid < 4 || (wid >= 6 && wid < 10)) {
       // ---- correction + epilogue: thread = query row.  Warps 6-9 are the partners of warps 2, 3, 0, 1 (same
-      // tensor-memory lanes): each of a pair rescales one half of the row's 512 columns.  Epilogue: warps 0-3.
+      // tensor-memory lanes): each of a pair takes one half of the row's 512 columns, in the rescale and in the epilogue.
       const bool partner = wid >= 4;
       const int r = (wid & 3) * 32 + lane;
       const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
@@ -686,7 +685,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       while (ok && iter.next(u)) {
         const int npages = 2 * (u.t1 - u.t0);
         int2 info;
-        const int slot = partner ? -1 : iter.slot_of(u, &info);
+        const int slot = iter.slot_of(u, &info);
         if (tid == 0 && leader) prm.item_info[u.it] = info;
         float inv = 0.f, lse = 0.f;
         for (int pi = 0; pi < npages && ok; ++pi, ++gt) {
@@ -696,7 +695,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           if (tid == 0) QSTAMP(smem_base, 6, gt);
           const uint32_t pbuf = smem_base + kOffP + s * kPStride;
           const uint32_t nword = ld_shared_b32(pbuf + kNOff + r * 4);
-          if (pi + 1 == npages && !partner) {
+          if (pi + 1 == npages) {
             uint32_t x, y;
             asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(pbuf + kFinOff + r * 8));
             inv = __uint_as_float(x); lse = __uint_as_float(y);
@@ -752,67 +751,49 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           if (tid == 0) QSTAMP(smem_base, 7, gt);
         }
         if (!ok) break;
-        // ---- epilogue (line 20): out = O / (l * S16)
-        if (!partner) {
+        // ---- epilogue (line 20): out = O / (l * S16).  Thread = row; a warp and its partner take eight 32-column
+        // chunks each, scale them and store them from registers with 256-bit stores (a full 32-byte sector per lane).
+        {
           const uint32_t gl = gt - 1;
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
           tc_fence_after_sync();
           if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 10 + 4 * un); };
-          const int row0 = u.r0 + half * kRowBlock;               // first row of this CTA within the sequence
-          const bool valid = row0 + r < prm.R;
-          const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
-          const int rows_here = min(32, prm.R - row0 - wid * 32);
-          __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + row0 + wid * 32) * kDv;
-          float* pbase = prm.part_o + (static_cast<size_t>(slot < 0 ? 0 : slot) * kItemRows + half * kRowBlock + wid * 32) * kDv;
+          const int row = u.r0 + half * kRowBlock + r;               // this thread's row within the sequence
+          const bool valid = row < prm.R;
+          __nv_bfloat16* orow = prm.out + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDv;
+          float* prow = prm.part_o + (static_cast<size_t>(slot < 0 ? 0 : slot) * kItemRows + half * kRowBlock + r) * kDv;
           uint32_t o[2][32];
-          tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
+          tmem_ld_32x32b_x32(tbase + lane_base + 32 * c_first, o[0]);
 #pragma unroll 1
-          for (int cq = 0; cq < 16; cq += 2) {
+          for (int cq = 0; cq < 8; cq += 2) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               tmem_wait_ld();
-              if (cq + e + 1 < 16) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (cq + e + 1), o[e ^ 1]);
-              const int cc = cq + e;
-              __syncwarp();
+              if (cq + e + 1 < 8) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (c_first + cq + e + 1), o[e ^ 1]);
+              const int cc = c_first + cq + e;
               if (slot < 0) {
+                uint32_t w[16];
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                  const uint32_t w0 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 0]) * inv, __uint_as_float(o[e][8 * jj + 1]) * inv);
-                  const uint32_t w1 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 2]) * inv, __uint_as_float(o[e][8 * jj + 3]) * inv);
-                  const uint32_t w2 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 4]) * inv, __uint_as_float(o[e][8 * jj + 5]) * inv);
-                  const uint32_t w3 = pack_bf16x2(__uint_as_float(o[e][8 * jj + 6]) * inv, __uint_as_float(o[e][8 * jj + 7]) * inv);
-                  st_shared_v4(epi + lane * 128 + ((jj ^ (lane & 7)) << 4), w0, w1, w2, w3);
+                for (int jj = 0; jj < 16; ++jj)
+                  w[jj] = pack_bf16x2(__uint_as_float(o[e][2 * jj]) * inv, __uint_as_float(o[e][2 * jj + 1]) * inv);
+                if (valid) {
+                  stg_256(orow + 32 * cc, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                  stg_256(orow + 32 * cc + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
                 }
-                __syncwarp();
+              } else if (valid) {
 #pragma unroll
-                for (int kq = 0; kq < 4; ++kq) {                       // 8 rows x 64 B per instruction
-                  const int row = 8 * kq + (lane >> 2), jj = lane & 3;
-                  uint4 v;
-                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                               : "r"(epi + row * 128 + ((jj ^ (row & 7)) << 4)));
-                  if (row < rows_here) *reinterpret_cast<uint4*>(obase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * jj) = v;
-                }
-              } else {
-#pragma unroll
-                for (int jj = 0; jj < 8; ++jj)
-                  st_shared_v4(epi + lane * 128 + ((jj ^ (lane & 7)) << 4),
-                               __float_as_uint(__uint_as_float(o[e][4 * jj + 0]) * inv), __float_as_uint(__uint_as_float(o[e][4 * jj + 1]) * inv),
-                               __float_as_uint(__uint_as_float(o[e][4 * jj + 2]) * inv), __float_as_uint(__uint_as_float(o[e][4 * jj + 3]) * inv));
-                __syncwarp();
-#pragma unroll
-                for (int kq = 0; kq < 8; ++kq) {                       // 4 rows x 128 B per instruction
-                  const int row = 4 * kq + (lane >> 3), jj = lane & 7;
-                  uint4 v;
-                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                               : "r"(epi + row * 128 + ((jj ^ (row & 7)) << 4)));
-                  if (row < rows_here) *reinterpret_cast<uint4*>(pbase + static_cast<size_t>(row) * kDv + 32 * cc + 4 * jj) = v;
-                }
+                for (int jj = 0; jj < 4; ++jj)
+                  stg_256(prow + 32 * cc + 8 * jj,
+                          __float_as_uint(__uint_as_float(o[e][8 * jj + 0]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 1]) * inv),
+                          __float_as_uint(__uint_as_float(o[e][8 * jj + 2]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 3]) * inv),
+                          __float_as_uint(__uint_as_float(o[e][8 * jj + 4]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 5]) * inv),
+                          __float_as_uint(__uint_as_float(o[e][8 * jj + 6]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 7]) * inv));
               }
             }
           }
-          if (valid) {
-            if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + row0 + r] = lse;
+          if (valid && !partner) {
+            if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + row] = lse;
             else prm.part_lse[static_cast<size_t>(slot) * kItemRows + half * kRowBlock + r] = lse;
           }
           tc_fence_before_sync();
