@@ -19,6 +19,27 @@ def _dense(w, b=0):
     return q, kv, kv[:, :512]
 
 
+# ---------------------------------------------------------------- bf16 rounding used by the simulators
+
+def test_bf16_round_ties_and_carries_by_hand():
+    f = lambda bits: np.array([bits], np.uint32).view(np.float32)
+    cases = [
+        (0x3F800000, 0x3F800000),   # 1.0 is representable
+        (0x3F808000, 0x3F800000),   # 1 + 2^-8: exactly half way between 1 and 1 + 2^-7 -> even (1.0)
+        (0x3F818000, 0x3F820000),   # 1 + 3 * 2^-8... half way between 0x3F81 and 0x3F82 -> even (0x3F82)
+        (0x3F808001, 0x3F810000),   # just above the half way point -> up
+        (0x3F80C000, 0x3F810000),   # 1 + 3 * 2^-9 -> nearest is 1 + 2^-7
+        (0x3F807FFF, 0x3F800000),   # just below half way -> down
+        (0x3FFFFFFF, 0x40000000),   # mantissa carry into the exponent: 1.9999999 -> 2.0
+        (0x7F7FFFFF, 0x7F800000),   # the largest finite float rounds to +inf in bf16
+        (0xBF808000, 0xBF800000),   # sign is carried along
+        (0x00000000, 0x00000000),
+    ]
+    for src, want in cases:
+        got = S.bf16_round(f(src)).view(np.uint32)[0]
+        assert got == want, (hex(src), hex(got), hex(want))
+
+
 # ---------------------------------------------------------------- Lemma 3.1
 
 def test_example_3_1_bit_pattern():

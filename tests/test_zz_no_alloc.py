@@ -4,15 +4,17 @@ A serving loop that must stay out of the allocator, a process whose device memor
 start-up, or a plugin that only ever receives input and output buffers cannot provide the workspace that
 amla_mla_decode asks for.  The static entry point runs the same kernels on a scratch array built into the library.
 This test calls it through the C-ABI twice in a row, on two different problems (so the second call finds the first
-call's leftovers in the shared scratch), and checks each result against the ordinary entry point within the
-tolerances of the parity tests.  The file name sorts last on purpose: a run that stops at the first failure has
+call's leftovers in the shared scratch), and checks each result against the ordinary entry point and against the
+FP64 oracle within the tolerances of the parity tests; the status word of the built-in scratch is read back after
+each call.  The file name sorts last on purpose: a run that stops at the first failure has
 then already executed every other test.
 """
 import numpy as np
 import pytest
 
+from oracle import reference as R
 from paper_2509_25224_b200 import binding, synth
-from tests._gpu_util import TOL_ABS, TOL_LSE, TOL_REL_L2, to_device
+from tests._gpu_util import TOL_ABS, TOL_LSE, TOL_REL_L2, compare, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -31,6 +33,7 @@ def _both(w):
     lse.fill_(float("nan"))
     torch.cuda.synchronize()
     binding.mla_decode_static(q, kv, bt, sl, w.scale, out, lse)
+    binding.static_check_status()          # no bounded wait ran out inside the static call
     torch.cuda.synchronize()
     return (out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64),
             ref_o.float().cpu().numpy().astype(np.float64), ref_l.cpu().numpy().astype(np.float64))
@@ -45,6 +48,9 @@ def _check(w):
     assert np.array_equal(np.isneginf(l), inf)
     if (~inf).any():
         assert np.abs(l[~inf] - rl[~inf]).max() <= TOL_LSE
+    # and against the FP64 oracle (CUDA against CUDA alone would not notice an error both entry points share)
+    oo, ol = R.decode(w.q, w.kv, w.block_table, w.seqlens, w.scale)
+    compare(o, l, oo, ol, "static entry vs oracle")
 
 
 def test_static_entry_matches_workspace_entry_on_two_calls_in_a_row():
