@@ -339,6 +339,7 @@ def run_gpu(args):
             per_config[w.name + " tau=0"] = entry(run, w, tau0)
         del run
         torch.cuda.empty_cache()
+        per_config["dsv3 fp8-cache"] = fp8_entry(synth.CONFIGS["dsv3"]() if w.name != "dsv3" else w, dev, local, ksteps, barrier, peaks, peak_kind)
         for name in synth.CONFIGS:
             if name == w.name:
                 continue
@@ -376,6 +377,43 @@ def run_gpu(args):
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+def fp8_entry(w, dev, local, steps, barrier, peaks, peak_kind, kv_scale=1.0 / 64.0):
+    """The same workload with an E4M3 cache (amla_mla_decode_fp8: widen the used pages, then the bf16 kernels): whole
+    call, CUDA events; its algorithmic bytes count one byte per cache element."""
+    import torch
+    from paper_2509_25224_b200 import binding
+    kv8 = synth.quantise_cache_e4m3(w, kv_scale)
+    q = torch.from_numpy(w.q.view(np.int16)).to(dev).view(torch.bfloat16)
+    bt, sl = torch.from_numpy(w.block_table).to(dev), torch.from_numpy(w.seqlens).to(dev)
+    caches = [torch.from_numpy(kv8).to(dev) for _ in range(max(2, int(np.ceil(200e6 / kv8.nbytes))))]
+    out = torch.empty((w.B, w.Sq, w.H, 512), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((w.B, w.Sq, w.H), dtype=torch.float32, device=dev)
+    ws = torch.empty(binding.fp8_workspace_size(w.B, w.Sq, w.H, w.max_blocks_per_seq, local), dtype=torch.uint8, device=dev)
+    for i in range(5):
+        binding.mla_decode_fp8(q, caches[i % len(caches)], kv_scale, bt, sl, w.scale, out, lse, ws)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    evs[0].record()
+    for i in range(steps):
+        binding.mla_decode_fp8(q, caches[i % len(caches)], kv_scale, bt, sl, w.scale, out, lse, ws)
+        evs[i + 1].record()
+    barrier()
+    binding.check_status(ws)
+    tot = evs[0].elapsed_time(evs[-1])
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+    flops = w.flops()
+    rows = w.B * w.Sq * w.H
+    alg_bytes = float(w.seqlens.astype(np.int64).sum()) * synth.D_QK + rows * synth.D_QK * 2 + rows * (synth.D_V * 2 + 4)
+    ms = tot / steps
+    t_b, t_f = alg_bytes / (float(peaks["hbm_gbs"]) * 1e9), flops / (float(peaks["bf16_tflops"]) * 1e12)
+    bound = "hbm" if t_b >= t_f else "tensor"
+    frac = max(t_b, t_f) / (ms * 1e-3)
+    return {"ms_per_step": ms, "median_step_ms": statistics.median(per), "tflops": flops / (ms * 1e-3) / 1e12, "bound": bound,
+            "frac": frac, "frac_of": "whole call (widen + decode + combine) against the " + peak_kind + " peak", "steps": steps,
+            "algorithmic_bytes": alg_bytes, "launches_per_step": binding.last_launch_count(),
+            "workload": workload_name(w).replace("bf16 paged-64", "bf16 q, E4M3 cache (scale 1/64) paged-64")}
 
 
 def load_traffic():

@@ -142,6 +142,29 @@ int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block
                        int num_blocks, int max_blocks_per_seq, void* out, float* lse, void* workspace,
                        size_t workspace_bytes, void* cuda_stream, int flags);
 
+/*
+ * The same decode on an FP8 cache (the remark after Lemma 3.1: the rescaling trick is tied to the accumulator's
+ * format, not to the inputs'; the accumulator stays FP32, Q and P~ stay bf16).
+ *
+ *   kv_cache_e4m3  device, uint8 [num_blocks, 64, 576], 16-byte aligned: OCP FP8 E4M3 (1 sign, 4 exponent bits with
+ *                  bias 7, 3 mantissa bits; no infinities, S.1111.111 is NaN).  The value of an element is
+ *                  decode(byte) * kv_scale; its first 512 columns are V.  Page layout and block table as above.
+ *   kv_scale       one dequantisation factor for the whole cache
+ *   workspace      at least amla_mla_decode_fp8_workspace_size() bytes, 256-byte aligned
+ *   flags          as for amla_mla_decode_ex
+ *
+ * Two passes: the pages the batch uses are first widened, exactly, into a bf16 copy inside the workspace
+ * (B * max_blocks_per_seq pages of 73 728 bytes), kv_scale is folded into the softmax scale and into the final
+ * normalisation, and the bf16 kernels run on the copy.  The FP8 cache saves device memory, not traffic: a call reads
+ * the FP8 pages and writes and reads their copy.  Everything else (visibility rule, outputs, errors) is as for
+ * amla_mla_decode.  A block-table entry outside [0, num_blocks) of a used page reads as a page of zeros.
+ */
+int amla_mla_decode_fp8_workspace_size(int B, int Sq, int H, int max_blocks_per_seq, int device, size_t* bytes_out);
+int amla_mla_decode_fp8(const void* q, const void* kv_cache_e4m3, float kv_scale, const int32_t* block_table,
+                        const int32_t* seqlens, float softmax_scale, int B, int Sq, int H, int num_blocks,
+                        int max_blocks_per_seq, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream, int flags);
+
 /* Synchronises `cuda_stream` and reads the status word the kernels keep at the start of the
  * workspace: AMLA_OK, or AMLA_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel expired (the
  * kernel then returned early and the outputs are undefined).  Optional. */

@@ -37,7 +37,7 @@ EXPORTS = [
     "amla_status_string", "amla_mla_decode_workspace_size", "amla_mla_decode", "amla_mla_decode_ex",
     "amla_check_status", "amla_last_launch_count", "amla_plan_host", "amla_profile_enable",
     "amla_profile_last_ms", "amla_mla_decode_static", "amla_static_check_status", "amla_wait_selftest",
-    "amla_validate_paging_host",
+    "amla_validate_paging_host", "amla_mla_decode_fp8", "amla_mla_decode_fp8_workspace_size",
 ]
 
 _lib = None
@@ -67,6 +67,10 @@ def lib() -> ctypes.CDLL:
         L.amla_mla_decode.restype = i32
         L.amla_mla_decode_ex.argtypes = dec + [i32]
         L.amla_mla_decode_ex.restype = i32
+        L.amla_mla_decode_fp8_workspace_size.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
+        L.amla_mla_decode_fp8_workspace_size.restype = i32
+        L.amla_mla_decode_fp8.argtypes = [vp, vp, f32, vp, vp, f32, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp, i32]
+        L.amla_mla_decode_fp8.restype = i32
         L.amla_mla_decode_static.argtypes = [vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, vp, vp, vp]
         L.amla_mla_decode_static.restype = i32
         L.amla_static_check_status.argtypes = [vp]
@@ -145,6 +149,47 @@ def mla_decode_static(q, kv_cache, block_table, seqlens, softmax_scale: float, o
                                           out.data_ptr(), lse.data_ptr(), stream)
     if rc != AMLA_OK:
         raise AmlaError(rc, "amla_mla_decode_static")
+
+
+def fp8_workspace_size(B: int, Sq: int, H: int, max_blocks_per_seq: int, device: int = 0) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().amla_mla_decode_fp8_workspace_size(B, Sq, H, max_blocks_per_seq, device, ctypes.byref(n))
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_mla_decode_fp8_workspace_size")
+    return int(n.value)
+
+
+def mla_decode_fp8(q, kv_cache_e4m3, kv_scale: float, block_table, seqlens, softmax_scale: float, out=None, lse=None,
+                   workspace=None, flags: int | None = None):
+    """amla_mla_decode_fp8 on device tensors: q bf16 [B,Sq,H,576], kv_cache_e4m3 uint8 [num_blocks,64,576] (E4M3 bytes;
+    element value = decode(byte) * kv_scale).  Returns (out bf16, lse fp32)."""
+    import torch
+
+    if kv_cache_e4m3.dtype != torch.uint8 or q.dtype != torch.bfloat16:
+        raise ValueError("q must be bfloat16 and the cache uint8 (E4M3 bytes)")
+    if block_table.dtype != torch.int32 or seqlens.dtype != torch.int32:
+        raise ValueError("block_table and seqlens must be int32")
+    if not (q.is_contiguous() and kv_cache_e4m3.is_contiguous() and block_table.is_contiguous() and seqlens.is_contiguous()):
+        raise ValueError("inputs must be contiguous")
+    B, Sq, H, d = q.shape
+    if d != 576 or tuple(kv_cache_e4m3.shape[1:]) != (64, 576) or block_table.shape[0] != B or seqlens.shape[0] != B:
+        raise ValueError("shape mismatch")
+    dev = q.device
+    if out is None:
+        out = torch.empty((B, Sq, H, 512), dtype=torch.bfloat16, device=dev)
+    if lse is None:
+        lse = torch.empty((B, Sq, H), dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(fp8_workspace_size(B, Sq, H, block_table.shape[1], dev.index or 0), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    with torch.cuda.device(dev):
+        rc = lib().amla_mla_decode_fp8(q.data_ptr(), kv_cache_e4m3.data_ptr(), float(kv_scale), block_table.data_ptr(),
+                                       seqlens.data_ptr(), float(softmax_scale), B, Sq, H, kv_cache_e4m3.shape[0],
+                                       block_table.shape[1], out.data_ptr(), lse.data_ptr(), workspace.data_ptr(),
+                                       workspace.numel(), stream, DEFAULT_FLAGS if flags is None else int(flags))
+    if rc != AMLA_OK:
+        raise AmlaError(rc, "amla_mla_decode_fp8")
+    return out, lse
 
 
 def static_check_status(stream: int = 0) -> None:

@@ -15,6 +15,8 @@ cudaError_t launch_decode_simt(const DecodeParams& prm, cudaStream_t stream);
 cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* unsupported);
 cudaError_t launch_decode_quad(const DecodeParams& prm, cudaStream_t stream, int* unsupported);
 cudaError_t launch_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t stream);
+cudaError_t launch_widen_pages(const uint8_t* kv8, const int32_t* block_table, const int32_t* seqlens, int B, int num_blocks,
+                               int max_blocks_per_seq, __nv_bfloat16* scratch, int32_t* table_out, cudaStream_t stream);
 int decode_tc_parts(int sm_count);
 int decode_quad_parts(int device, int sm_count);
 
@@ -166,11 +168,13 @@ extern "C" int amla_mla_decode_workspace_size(int B, int Sq, int H, int max_bloc
   return AMLA_OK;
 }
 
-extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block_table,
-                                  const int32_t* seqlens, float softmax_scale, int B, int Sq, int H,
-                                  int num_blocks, int max_blocks_per_seq, void* out, float* lse,
-                                  void* workspace, size_t workspace_bytes, void* cuda_stream, int flags) {
-  g_last_launches = 0;
+namespace {
+
+// The decode call on a bf16 cache.  out_scale multiplies the normalised output (1 unless the cache was widened from
+// FP8 with a dequantisation scale); launches are added to g_last_launches.
+int decode_impl(const void* q, const void* kv_cache, const int32_t* block_table, const int32_t* seqlens,
+                float softmax_scale, float out_scale, int B, int Sq, int H, int num_blocks, int max_blocks_per_seq,
+                void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream, int flags) {
   if (!q || !kv_cache || !block_table || !seqlens || !out || !lse || !workspace) return AMLA_ERR_INVALID_ARG;
   if (num_blocks <= 0 || !(softmax_scale == softmax_scale)) return AMLA_ERR_INVALID_ARG;
   int rc = check_shape(B, Sq, H, max_blocks_per_seq);
@@ -209,6 +213,7 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   prm.part_lse = reinterpret_cast<float*>(ws + lay.part_lse_off);
   prm.part_o = reinterpret_cast<float*>(ws + lay.part_o_off);
   prm.scale_log2 = softmax_scale * kLog2e;
+  prm.out_scale = out_scale;
   prm.B = B; prm.Sq = Sq; prm.H = H;
   prm.R = Sq * H;
   prm.num_blocks = num_blocks;
@@ -221,6 +226,64 @@ extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int
   rc = configure_schedule(prm, device, sms, flags);
   if (rc != AMLA_OK) return rc;
   return launch_decode_call(prm, prefix, static_cast<cudaStream_t>(cuda_stream), &g_last_launches, profile_mark);
+}
+
+// Bytes of the FP8 path's extra scratch behind the ordinary workspace: the new block table and the widened pages.
+size_t fp8_table_bytes(int B, int max_blocks_per_seq) { return align_up(sizeof(int32_t) * static_cast<size_t>(B) * max_blocks_per_seq); }
+size_t fp8_pages_bytes(int B, int max_blocks_per_seq) { return static_cast<size_t>(B) * max_blocks_per_seq * kPage * kDqk * sizeof(__nv_bfloat16); }
+
+}  // namespace
+
+extern "C" int amla_mla_decode_ex(const void* q, const void* kv_cache, const int32_t* block_table,
+                                  const int32_t* seqlens, float softmax_scale, int B, int Sq, int H,
+                                  int num_blocks, int max_blocks_per_seq, void* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream, int flags) {
+  g_last_launches = 0;
+  return decode_impl(q, kv_cache, block_table, seqlens, softmax_scale, 1.f, B, Sq, H, num_blocks, max_blocks_per_seq, out, lse,
+                     workspace, workspace_bytes, cuda_stream, flags);
+}
+
+extern "C" int amla_mla_decode_fp8_workspace_size(int B, int Sq, int H, int max_blocks_per_seq, int device, size_t* bytes_out) {
+  size_t base = 0;
+  const int rc = amla_mla_decode_workspace_size(B, Sq, H, max_blocks_per_seq, device, &base);
+  if (rc != AMLA_OK) return rc;
+  *bytes_out = align_up(base) + fp8_table_bytes(B, max_blocks_per_seq) + fp8_pages_bytes(B, max_blocks_per_seq);
+  return AMLA_OK;
+}
+
+extern "C" int amla_mla_decode_fp8(const void* q, const void* kv_cache_e4m3, float kv_scale, const int32_t* block_table,
+                                   const int32_t* seqlens, float softmax_scale, int B, int Sq, int H, int num_blocks,
+                                   int max_blocks_per_seq, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream, int flags) {
+  g_last_launches = 0;
+  if (!q || !kv_cache_e4m3 || !block_table || !seqlens || !out || !lse || !workspace) return AMLA_ERR_INVALID_ARG;
+  if (num_blocks <= 0 || !(kv_scale == kv_scale) || !(softmax_scale == softmax_scale)) return AMLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(kv_cache_e4m3) & 15) return AMLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) return AMLA_ERR_INVALID_ARG;
+  int rc = check_shape(B, Sq, H, max_blocks_per_seq);
+  if (rc != AMLA_OK) return rc;
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return AMLA_ERR_CUDA; }
+  size_t base = 0;
+  rc = amla_mla_decode_workspace_size(B, Sq, H, max_blocks_per_seq, device, &base);
+  if (rc != AMLA_OK) return rc;
+  base = align_up(base);
+  const size_t tbytes = fp8_table_bytes(B, max_blocks_per_seq), pbytes = fp8_pages_bytes(B, max_blocks_per_seq);
+  if (workspace_bytes < base + tbytes + pbytes) return AMLA_ERR_WORKSPACE;
+  if (static_cast<long long>(B) * max_blocks_per_seq > (1ll << 30)) return AMLA_ERR_UNSUPPORTED;
+  char* ws = static_cast<char*>(workspace);
+  int32_t* table2 = reinterpret_cast<int32_t*>(ws + base);
+  __nv_bfloat16* pages = reinterpret_cast<__nv_bfloat16*>(ws + base + tbytes);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (launch_widen_pages(static_cast<const uint8_t*>(kv_cache_e4m3), block_table, seqlens, B, num_blocks, max_blocks_per_seq,
+                         pages, table2, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return AMLA_ERR_CUDA;
+  }
+  ++g_last_launches;
+  // logits: scale * q . (k8 * kv_scale); output: sum p * (v8 * kv_scale)
+  return decode_impl(q, pages, table2, seqlens, softmax_scale * kv_scale, kv_scale, B, Sq, H, B * max_blocks_per_seq,
+                     max_blocks_per_seq, out, lse, workspace, base, cuda_stream, flags);
 }
 
 extern "C" int amla_mla_decode(const void* q, const void* kv_cache, const int32_t* block_table,

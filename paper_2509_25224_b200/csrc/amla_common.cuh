@@ -34,6 +34,7 @@ struct DecodeParams {
                                  // the decode kernel for every item it touches, read by the combine
   float scale_log2;              // softmax_scale * log2(e)
   float tau;                     // lazy-reference threshold in octaves (0 = move the reference with every new maximum)
+  float out_scale;               // factor on the normalised output (1; the dequantisation scale of an FP8 cache's V)
   int B, Sq, H;
   int R;                         // Sq * H query rows per sequence
   int nrb;                       // row blocks per sequence = ceil(R / 128)

@@ -366,7 +366,7 @@ __device__ __noinline__ uint32_t softmax_unit(const DecodeParams prm, const Role
         const float l_all = st.l + exchange(st.l);
         if (ok && hsel == 1) {
           const bool live = l_all > 0.f;
-          const float inv = live ? 1.f / (l_all * st.s_out) : 0.f;
+          const float inv = live ? prm.out_scale / (l_all * st.s_out) : 0.f;
           const float lse = live ? (st.m2 + log2f(l_all)) * kLn2 : -INFINITY;
           st_async_v2(dstp + kFinOff + r * 8, __float_as_uint(inv), __float_as_uint(lse), pfull);
         }

@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
         const int row = pass * kRowsPerPass + wid * kRowsPerWarp + rr;
         if (row >= nrows) continue;
         const bool live = st[rr].l > 0.f;
-        const float inv = live ? 1.f / (st[rr].l * st[rr].s_out) : 0.f;
+        const float inv = live ? prm.out_scale / (st[rr].l * st[rr].s_out) : 0.f;
         const float lse = live ? (st[rr].m2 + log2f(st[rr].l)) * kLn2 : -INFINITY;
         if (slot < 0) {
           __nv_bfloat16* orow = prm.out + (static_cast<size_t>(b) * prm.R + r0 + row) * kDv;

@@ -359,7 +359,7 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
     if (ok) ok = warp_wait<true>(bar(A_FINFREE + (un & 1)), ((un >> 1) & 1) ^ 1);
     if (ok) {
       const bool live = st.l > 0.f;
-      const float inv = live ? 1.f / (st.l * st.s_out) : 0.f;
+      const float inv = live ? prm.out_scale / (st.l * st.s_out) : 0.f;
       const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
       // asynchronous remote stores counted on the barrier: no thread has to wait for a cluster-scope release
       const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;

@@ -118,6 +118,7 @@ extern "C" int amla_mla_decode_static(const void* q, const void* kv_cache, const
   prm.part_lse = reinterpret_cast<float*>(ws + kPartLseOff);
   prm.part_o = reinterpret_cast<float*>(ws + kPartOOff);
   prm.scale_log2 = softmax_scale * kLog2e;
+  prm.out_scale = 1.f;
   prm.B = B; prm.Sq = Sq; prm.H = H;
   prm.R = Sq * H;
   prm.num_blocks = num_blocks;

@@ -46,6 +46,32 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def f32_to_e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to OCP FP8 E4M3 (nearest even, saturating at +-448); returns the uint8 bit patterns.
+    Input preparation for the FP8-cache workloads: 1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits; exponent
+    field 0 holds the subnormals m * 2^-9; S.1111.111 (NaN) is never produced."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    sign = (np.signbit(x)).astype(np.uint8) << 7
+    a = np.minimum(np.abs(x).astype(np.float64), 448.0)
+    # spacing of the E4M3 grid at |x|: 2^(e-3) with e = max(floor(log2 |x|), -6)
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)
+    step = np.exp2(e - 3.0)
+    k = np.rint(a / step)                 # nearest even multiple count (numpy rounds half to even)
+    v = k * step                          # may land on the next binade (k = 16), still representable or 448+ -> clamp
+    v = np.minimum(v, 448.0)
+    # encode v exactly
+    with np.errstate(divide="ignore"):
+        ev = np.floor(np.log2(np.where(v > 0, v, 1.0)))
+    ev = np.maximum(ev, -6.0)
+    mant = v / np.exp2(ev)                # in [1, 2) for normals, [0, 1) for subnormals
+    is_sub = v < 2.0 ** -6
+    efield = np.where(is_sub, 0, ev + 7).astype(np.int64)
+    mfield = np.where(is_sub, np.rint(v * 512.0), np.rint((mant - 1.0) * 8.0)).astype(np.int64)
+    return (sign | (efield.astype(np.uint8) << 3) | mfield.astype(np.uint8)).astype(np.uint8)
+
+
 @dataclass
 class Workload:
     name: str
@@ -127,6 +153,20 @@ def make_workload(name: str, B: int, Sq: int, H: int, seqlens, seed: int, *,
         off += k
     return Workload(name, B, Sq, H, seqlens, q, kv, bt, float(scale),
                     meta={"seed": seed, "dist": dist, "sigma": sigma, "shuffled": shuffle_pages})
+
+
+def quantise_cache_e4m3(w: Workload, kv_scale: float = 1.0 / 64.0) -> np.ndarray:
+    """uint8 [num_blocks, 64, 576]: the workload's bf16 cache divided by kv_scale and rounded to E4M3 (the FP8-cache
+    variant of the same workload; element value = decode(byte) * kv_scale).  With the default scale N(0,1) values
+    land around +-64 in the E4M3 range (max 448)."""
+    out = np.empty(w.kv.shape, dtype=np.uint8)
+    flat_in = w.kv.reshape(-1)
+    flat_out = out.reshape(-1)
+    chunk = 1 << 24
+    for s0 in range(0, flat_in.size, chunk):
+        x = bf16_bits_to_f32(flat_in[s0:s0 + chunk]) / np.float32(kv_scale)
+        flat_out[s0:s0 + chunk] = f32_to_e4m3_bits(x)
+    return out
 
 
 def logical_kv_rows(w: Workload, b: int) -> np.ndarray:

@@ -79,6 +79,36 @@ def test_bounded_wait_reports_a_timeout_instead_of_hanging():
     check_full(synth.config_tiny())
 
 
+def _check_fp8(w, kv_scale=1.0 / 64.0, flags=None):
+    import torch
+    from tests._gpu_util import compare
+    kv8 = synth.quantise_cache_e4m3(w, kv_scale)
+    ro, rl = R.decode_fp8(w.q, kv8, kv_scale, w.block_table, w.seqlens, w.scale)
+    q, _, bt, sl = to_device(w)
+    kvd = torch.from_numpy(kv8).to(q.device)
+    out = torch.empty((w.B, w.Sq, w.H, 512), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((w.B, w.Sq, w.H), dtype=torch.float32, device=q.device)
+    ws = torch.empty(binding.fp8_workspace_size(w.B, w.Sq, w.H, bt.shape[1], 0), dtype=torch.uint8, device=q.device)
+    out.view(torch.int16).fill_(0x7FC0); lse.fill_(float("nan")); ws.fill_(0xFF)
+    binding.mla_decode_fp8(q, kvd, kv_scale, bt, sl, w.scale, out, lse, ws, flags)
+    binding.check_status(ws)
+    torch.cuda.synchronize()
+    return compare(out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64), ro, rl, "fp8 " + w.name)
+
+
+def test_fp8_cache_small_shapes():
+    # E4M3 cache with a per-tensor scale against the FP64 oracle on the same bytes: tiny, ragged with an empty
+    # sequence, two query tokens (256-row kernel), a scale that is not a power of two
+    _check_fp8(synth.config_tiny())
+    _check_fp8(synth.make_workload("f8r", 5, 1, 128, [700, 0, 64, 129, 1], seed=601))
+    _check_fp8(synth.make_workload("f8q", 3, 2, 128, [1000, 65, 300], seed=602), flags=binding.RESCALE_ALG2 | binding.lazy(0))
+    _check_fp8(synth.make_workload("f8s", 2, 1, 64, [500, 77], seed=603), kv_scale=0.0173)
+
+
+def test_fp8_cache_dsv3_shape_full():
+    _check_fp8(synth.config_dsv3())
+
+
 def test_all_sequences_empty():
     w = synth.make_workload("e", 3, 2, 128, [0, 0, 0], seed=7)
     out, lse, _ = run_gpu(w)

@@ -179,3 +179,52 @@ def test_flop_and_intensity_formulas_match_the_paper():
     # and synth.Workload.flops uses the same count
     w = synth.make_workload("t", 2, 2, 4, [10, 20], seed=1)
     assert w.flops() == 2.0 * 2 * 4 * 30 * 1088
+
+
+# ----------------------------------------------------------------- FP8 (E4M3) cache oracle
+
+def test_e4m3_widening_matches_the_library_conversion_on_all_bytes():
+    # the oracle's own decoder of OCP E4M3 bytes against torch's float8_e4m3fn on every byte value
+    import torch
+    b = torch.arange(256, dtype=torch.uint8)
+    want = b.view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    got = np.array([R.e4m3_to_double(i) for i in range(256)])
+    assert np.isnan(got[0x7F]) and np.isnan(got[0xFF]) and np.isnan(want[0x7F]) and np.isnan(want[0xFF])
+    ok = ~np.isnan(want)
+    assert ok.sum() == 254 and np.array_equal(got[ok], want[ok])
+    # a few values of the format by hand: 1.0, the largest (448), the smallest subnormal (2^-9), the smallest normal (2^-6), -1.5
+    assert got[0x38] == 1.0 and got[0x7E] == 448.0 and got[0x01] == 2.0 ** -9 and got[0x08] == 2.0 ** -6 and got[0xBC] == -1.5
+
+
+def test_e4m3_quantiser_of_the_input_generator():
+    import torch
+    # every representable value maps to its own byte ...
+    vals = np.array([R.e4m3_to_double(i) for i in range(256)])
+    ok = ~np.isnan(vals)
+    bits = synth.f32_to_e4m3_bits(vals[ok].astype(np.float32))
+    assert np.array_equal(bits, np.arange(256, dtype=np.uint8)[ok])
+    # ... in-range values round like the library's conversion (nearest even), out-of-range ones saturate at 448
+    rng = np.random.default_rng(3)
+    x = np.concatenate([rng.standard_normal(20000) * 60, rng.standard_normal(2000) * 0.01, [17.0, 19.0, 1.0625, 2.0 ** -10, 3 * 2.0 ** -10]]).astype(np.float32)
+    x = x[np.abs(x) <= 448]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = synth.f32_to_e4m3_bits(x)
+    nz = (want & 0x7F) != 0            # (the sign of a zero result is not compared)
+    assert np.array_equal(got[nz], want[nz]) and np.all((got[~nz] & 0x7F) == 0)
+    assert synth.f32_to_e4m3_bits(np.array([1e6, -1e6], np.float32)).tolist() == [0x7E, 0xFE]
+
+
+def test_fp8_oracle_equals_the_bf16_oracle_on_the_widened_cache():
+    # E4M3 values are exact in bf16, and a power-of-two scale keeps them exact: the FP8 oracle on (bytes, kv_scale)
+    # must agree with the bf16 oracle on the cache of widened, scaled values to rounding order
+    w = synth.make_workload("f8", 3, 2, 4, [130, 0, 65], seed=91)
+    for kv_scale in (1.0, 1.0 / 64.0):
+        kv8 = synth.quantise_cache_e4m3(w, kv_scale)
+        wide = np.array([R.e4m3_to_double(i) for i in range(256)])[kv8] * kv_scale
+        kv16 = synth.f32_to_bf16_bits(wide.astype(np.float32))
+        assert np.array_equal(synth.bf16_bits_to_f32(kv16).astype(np.float64), wide)      # exact in bf16
+        o8, l8 = R.decode_fp8(w.q, kv8, kv_scale, w.block_table, w.seqlens, w.scale)
+        o16, l16 = R.decode(w.q, kv16, w.block_table, w.seqlens, w.scale)
+        fin = ~np.isneginf(l16)
+        assert np.array_equal(np.isneginf(l8), ~fin)
+        assert np.abs(o8 - o16).max() <= 1e-12 and np.abs(l8[fin] - l16[fin]).max() <= 1e-12
