@@ -49,8 +49,8 @@ constexpr uint32_t kKSlotBytes = 3 * kBoxBytes;      // 64 keys x 192 columns: [
 constexpr uint32_t kKGroupStride = 3 * 1024;
 constexpr uint32_t kOffQRope = 0;                    // 128 rows x 64 bf16, 128-byte swizzle
 constexpr uint32_t kOffXchg = 128 * 64 * 2;          // float [2 exchanges in flight][2 warpgroups][128 rows]: what the two threads of a row tell each other
-constexpr uint32_t kOffStage = kOffXchg + 2 * 1024;  // 8 softmax warps x 4 KB: a warp's 32 rows of P~, in the byte order of the P buffer
-constexpr uint32_t kOffK = kOffStage + 8 * 4096;
+constexpr uint32_t kOffStage = kOffXchg + 2 * 1024;  // [2][8 softmax warps] x 4 KB: a warp's 32 rows of P~ in the byte order of the P buffer, two tiles in flight
+constexpr uint32_t kOffK = kOffStage + 2 * 8 * 4096;
 constexpr uint32_t kEndA = kOffK + kNumKSlots * kKSlotBytes;
 // ---- value CTA
 constexpr int kNumVSlots = 4;
@@ -61,14 +61,18 @@ constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;
 constexpr uint32_t kEndB = kOffP + kNumP * kPStride;
 // ---- all four: barriers at the same offset, so that one multicast commit reaches them
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
-constexpr uint32_t kBarBytes = 512;
-constexpr int kSmemPlanItems = 128;
+constexpr uint32_t kBarBytes = 256;
+#ifdef AMLA_TRACE
+constexpr int kSmemPlanItems = 4;                    // trace builds: the room goes to the stamps
+#else
+constexpr int kSmemPlanItems = 64;
+#endif
 constexpr uint32_t kOffPlan = kOffBars + kBarBytes;
 constexpr uint32_t kOffSeqlens = kOffPlan + ((kSmemPlanItems + 1) * 4 + 15) / 16 * 16;
 #ifdef AMLA_TRACE
 // trace builds: every CTA keeps its stamps (low 32 bits of its SM's cycle counter) in shared memory, so that taking
 // one does not put a global store in front of the role's next release, and dumps them when it is done
-constexpr int kQTraceEvents = 16, kQTraceIdx = 128;
+constexpr int kQTraceEvents = 16, kQTraceIdx = 11;
 constexpr uint32_t kOffTrace = kOffSeqlens + kSmemPlanItems * 4;
 constexpr uint32_t kSmemBytes = kOffTrace + kQTraceEvents * kQTraceIdx * 4;
 #define QSTAMP(smem_base_, ev, idx)                                                                          \
@@ -77,7 +81,11 @@ constexpr uint32_t kSmemBytes = kOffTrace + kQTraceEvents * kQTraceIdx * 4;
       st_shared_b32((smem_base_) + kOffTrace + ((ev) * kQTraceIdx + (idx)) * 4, static_cast<uint32_t>(clock64())); \
   } while (0)
 // event 15 holds wall-clock stamps (global timer, ns) of the kernel's phases, comparable across SMs and kernels
-#define QSTAMP_NS(smem_base_, idx) st_shared_b32((smem_base_) + kOffTrace + (15 * kQTraceIdx + (idx)) * 4, static_cast<uint32_t>(global_timer_ns()))
+#define QSTAMP_NS(smem_base_, idx)                                                                           \
+  do {                                                                                                       \
+    if (static_cast<unsigned>(idx) < static_cast<unsigned>(kQTraceIdx))                                      \
+      st_shared_b32((smem_base_) + kOffTrace + (15 * kQTraceIdx + (idx)) * 4, static_cast<uint32_t>(global_timer_ns())); \
+  } while (0)
 #else
 constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
 #define QSTAMP(smem_base_, ev, idx) do { } while (0)
@@ -331,32 +339,26 @@ __device__ __noinline__ uint32_t softmax_unit(const DecodeParams prm, const Role
         unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
         st.l = st.l * sp.l_up + __fdividef((rs0 + s0) + (rs1 + s1), sp.p_scale);   // this thread's share of the row sum
       }
-      // ---- ship the page: P~ (128 B of this row), the row's word N, and with the unit's last page the final scalars
-      const uint32_t stage = smem_base + kOffStage + (hsel * 4 + quarter) * 4096;
-#pragma unroll
-      for (int cc = 0; cc < 8; ++cc)
-        st_shared_v4(stage + sw128_offset(lane, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-      __syncwarp();
+      // ---- ship the page: P~ (128 B of this row), the row's word N, and with the unit's last page the final scalars.
+      // The warp's 32 rows are a contiguous 4 KB block of the P buffer: they are staged in a block of the warp's own
+      // and moved by the copy engine (remote stores by the threads would hold the warp at the rate of the SM-to-SM
+      // link, ~900 clk per tile).  Two staging blocks alternate; the one written now was last read for the page four
+      // pages back in the same P buffer, whose P V -- awaited next -- cannot have run before that copy had landed.
       const uint32_t gp = 2 * gs + hsel;                     // page number within the cluster's work
       const uint32_t pb = gp % kNumP;
       ok = warp_wait(bar(X_PV + pb), ((gp / kNumP) & 1) ^ 1);     // the P V that last read the buffer is done
       if (!ok) return;
+      const uint32_t stage = smem_base + kOffStage + ((gs & 1) * 8 + hsel * 4 + quarter) * 4096;
+#pragma unroll
+      for (int cc = 0; cc < 8; ++cc)
+        st_shared_v4(stage + sw128_offset(lane, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+      fence_proxy_async_smem();
+      __syncwarp();
       const bool with_fin = last_tile && hsel == 1;
       const uint32_t pfull = c.peer_bars + 8u * (B_PFULL + pb);
       const uint32_t dstp = c.peer_base + kOffP + pb * kPStride;
       if (quarter == 0 && lane == 0) { QSTAMP(c.smem_base, 5, gp); mbar_arrive_expect_tx_cluster(pfull, with_fin ? kPXferLast : kPXfer); }
-      // A thread's 128 bytes are eight 16-byte pieces of one row; sent as they are, every store instruction of the
-      // warp would be 32 separate small remote writes (measured: ~290 clk per instruction).  The warp's 32 rows are a
-      // contiguous 4 KB block of the P buffer, so it goes through a 4 KB staging block of the warp's own and leaves
-      // in instructions that cover 512 contiguous bytes each.
-      uint32_t v[8][4];
-#pragma unroll
-      for (int cc = 0; cc < 8; ++cc)
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[cc][0]), "=r"(v[cc][1]), "=r"(v[cc][2]), "=r"(v[cc][3])
-                     : "r"(stage + cc * 512 + lane * 16));
-#pragma unroll
-      for (int cc = 0; cc < 8; ++cc)
-        st_async_v4(dstp + quarter * 4096 + cc * 512 + lane * 16, v[cc][0], v[cc][1], v[cc][2], v[cc][3], pfull);
+      if (lane == 0) bulk_copy_to_cluster(dstp + quarter * 4096, stage, 4096, pfull);
       const uint32_t nword = (kMode == 2) ? __float_as_uint(hsel == 0 ? sp.l_up : 1.f)
                                           : static_cast<uint32_t>(hsel == 0 ? sp.n_bits : 0);
       st_async_b32(dstp + kNOff + r * 4, nword, pfull);
@@ -523,7 +525,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
         ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);      // the previous unit's QK^T is finished with Q
         if (!ok) break;
         tc_fence_after_sync();
-        if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 8 + 4 * un); };
+        if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 8 + 4 * un); };
         {
           const int row = u.r0 + half * kRowBlock + qr;
           const bool valid = row < prm.R;
@@ -541,7 +543,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
         }
         tc_fence_before_sync();
         warp_arrive(bar(A_QREADY), lane);
-        if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 9 + 4 * un); };
+        if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 9 + 4 * un); };
         if (grp_b) {                               // the next unit's Q goes to L2 while this one is computed
           UnitIter peek = iter;
           Unit nu;
@@ -758,7 +760,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
           tc_fence_after_sync();
-          if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 10 + 4 * un); };
+          if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 10 + 4 * un); };
           const int row = u.r0 + half * kRowBlock + r;               // this thread's row within the sequence
           const bool valid = row < prm.R;
           __nv_bfloat16* orow = prm.out + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDv;
@@ -797,7 +799,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             else prm.part_lse[static_cast<size_t>(slot) * kItemRows + half * kRowBlock + r] = lse;
           }
           tc_fence_before_sync();
-          if (tid == 0) { if (un < 20) QSTAMP_NS(smem_base, 11 + 4 * un); };
+          if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 11 + 4 * un); };
         }
         ++un;
       }
@@ -918,7 +920,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
   cluster_arrive();
   cluster_wait();
 #ifdef AMLA_TRACE
-  if (prm.trace && tid == 0) prm.trace[static_cast<size_t>(blockIdx.x) * kQTraceEvents * kQTraceIdx + 15 * kQTraceIdx + 7] = static_cast<uint32_t>(global_timer_ns());
+  if (prm.trace && tid == 0) prm.trace[static_cast<size_t>(blockIdx.x) * kQTraceEvents * kQTraceIdx + 15 * kQTraceIdx + 7] = static_cast<uint32_t>(global_timer_ns());   // idx 7 < kQTraceIdx
 #endif
   if (wid == 5) tmem_dealloc_pair(tbase, kTmemCols);
 }

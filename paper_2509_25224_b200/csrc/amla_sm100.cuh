@@ -161,6 +161,16 @@ __device__ __forceinline__ void tma_load_4d_pair(uint32_t dst_smem, const void* 
       ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(cluster_bar)
       : "memory");
 }
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster, carried out by the copy
+// engine (no thread waits for the link); the bytes are counted on a barrier of the destination CTA.  Both addresses
+// 16-byte aligned, size a multiple of 16.  Earlier generic-proxy writes to the source need fence.proxy.async first;
+// the source may be rewritten once the destination barrier's phase has completed.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(cluster_bar)
+      : "memory");
+}
 // 256-bit read-only global load (32-byte aligned address).
 __device__ __forceinline__ void ldg_256(const void* p, uint32_t (&r)[32], int at) {
   asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
