@@ -102,7 +102,7 @@ int configure_schedule(DecodeParams& prm, int device, int sms, int flags) {
   }
   prm.item_rows = quad ? 2 * kRowBlock : kRowBlock;
   prm.tile_keys = quad ? 2 * kPage : kPage;
-  prm.ovh = quad ? kUnitOverheadTiles / 2 : kUnitOverheadTiles;
+  prm.ovh = quad ? kQuadOverheadTiles : kUnitOverheadTiles;
   prm.nrb = (prm.R + prm.item_rows - 1) / prm.item_rows;
   prm.n_items = prm.B * prm.nrb;
   prm.P = simt ? sms : quad ? quad_parts : decode_tc_parts(sms);
@@ -370,7 +370,7 @@ extern "C" int amla_plan_host(const int32_t* seqlens, int B, int Sq, int H, int 
   if (rc != AMLA_OK) return rc;
   const bool quad = Sq * H > kRowBlock;
   const int item_rows = quad ? 2 * kRowBlock : kRowBlock, tile_keys = quad ? 2 * kPage : kPage;
-  const int ovh = quad ? kUnitOverheadTiles / 2 : kUnitOverheadTiles;
+  const int ovh = quad ? kQuadOverheadTiles : kUnitOverheadTiles;
   const int nrb = (Sq * H + item_rows - 1) / item_rows;
   const int n_items = B * nrb;
   int* prefix = new (std::nothrow) int[n_items + 1];

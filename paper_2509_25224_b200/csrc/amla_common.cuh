@@ -79,7 +79,11 @@ constexpr int kTraceTiles = 96;
 // L = prefix[n_items] the total, and part p owns positions [p*L/P, (p+1)*L/P).  A part does the
 // tiles whose positions it owns; overhead positions carry no work.
 // ---------------------------------------------------------------------------------------------
-constexpr int kUnitOverheadTiles = 10;        // in 64-key pages; halved when tiles are 128 keys
+constexpr int kUnitOverheadTiles = 10;        // 128-row kernel: in 64-key pages
+#ifndef AMLA_QUAD_OVERHEAD_TILES
+#define AMLA_QUAD_OVERHEAD_TILES 5            // 256-row kernel: in 128-key tiles (a build-time knob for tuning runs)
+#endif
+constexpr int kQuadOverheadTiles = AMLA_QUAD_OVERHEAD_TILES;
 constexpr int kFusedPlanMaxItems = 2048;   // up to this many items every decode CTA computes the prefix itself
 
 // Overhead positions in front of item `it`: none for the first item, which opens the first part anyway (every
