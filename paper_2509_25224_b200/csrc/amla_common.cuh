@@ -28,7 +28,8 @@ struct DecodeParams {
   float* lse;                    // [B, R]
   int* status;                   // workspace status word
   const int* prefix;             // [n_items + 1] linear tile index of each item's first tile
-  float* part_o;                 // [2 * P, 128, 512] fp32 normalised partial outputs
+  float* part_o;                 // normalised partial outputs of split items: [2 * P * item_rows][512] half precision, then
+                                 // [2 * P * item_rows][16] scale bytes (see "Split partials" below)
   float* part_lse;               // [2 * P, 128]      partial lse (natural log)
   int2* item_info;               // [n_items] (slot of the item's first partial, number of parts it is split over), written by
                                  // the decode kernel for every item it touches, read by the combine
@@ -159,6 +160,37 @@ struct Plan {
   // The same from what item_info holds: slot of split s (0 = the part where the item begins) of an item
   __host__ __device__ static int slot_of_split(int first_slot, int s) { return s == 0 ? first_slot : 2 * ((first_slot >> 1) + s); }
 };
+
+// ---------------------------------------------------------------------------------------------
+// Split partials.  A part that holds some of an item's tiles leaves the item's normalised output rows for the
+// combine kernel.  They travel in half precision (the combine rounds its result to bf16 anyway; a half has three
+// more mantissa bits), each 32-column chunk of a row scaled by a power of two so that its largest magnitude lies in
+// [1, 2): the chunk's scale byte is the biased FP32 exponent of that magnitude, the stored halves are value *
+// 2^(127 - byte), and value = half * 2^(byte - 127) exactly (byte 0: a chunk of zeros).  Half the bytes of FP32
+// partials, whatever the range of V.
+// ---------------------------------------------------------------------------------------------
+__host__ __device__ inline size_t partial_rows(const DecodeParams& prm) { return static_cast<size_t>(2) * prm.P * prm.item_rows; }
+__device__ __forceinline__ uint16_t* partial_halves(const DecodeParams& prm) { return reinterpret_cast<uint16_t*>(prm.part_o); }
+__device__ __forceinline__ uint8_t* partial_scales(const DecodeParams& prm) {
+  return reinterpret_cast<uint8_t*>(prm.part_o) + partial_rows(prm) * kDv * sizeof(uint16_t);
+}
+// scale byte and the factor 2^(127 - byte) for a chunk whose largest magnitude is max_abs
+__device__ __forceinline__ uint32_t partial_scale_byte(float max_abs, float* factor) {
+  const uint32_t e = min((__float_as_uint(max_abs) >> 23) & 0xffu, 253u);
+  *factor = __uint_as_float((254u - e) << 23);
+  return e;
+}
+__device__ __forceinline__ float partial_unscale(uint32_t scale_byte) { return __uint_as_float(scale_byte << 23); }
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float2 unpack_f16x2(uint32_t h2) {
+  float lo, hi;
+  asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.f32.f16 %0, a;\n\tcvt.f32.f16 %1, b;\n\t}" : "=f"(lo), "=f"(hi) : "r"(h2));
+  return make_float2(lo, hi);
+}
 
 // ---------------------------------------------------------------------------------------------
 // Lemma 3.1: F * 2^n == AS_FP32(AS_INT32(F) + n * 2^23) for normal F and 0 < E + n < 255.

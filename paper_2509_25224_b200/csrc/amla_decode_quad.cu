@@ -764,7 +764,9 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           const int row = u.r0 + half * kRowBlock + r;               // this thread's row within the sequence
           const bool valid = row < prm.R;
           __nv_bfloat16* orow = prm.out + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDv;
-          float* prow = prm.part_o + (static_cast<size_t>(slot < 0 ? 0 : slot) * kItemRows + half * kRowBlock + r) * kDv;
+          const size_t prow = static_cast<size_t>(slot < 0 ? 0 : slot) * kItemRows + half * kRowBlock + r;   // row of the partial arrays
+          uint16_t* hrow = partial_halves(prm) + prow * kDv;
+          uint32_t sc_lo = 0, sc_hi = 0;                                  // this thread's eight scale bytes
           uint32_t o[2][32];
           tmem_ld_32x32b_x32(tbase + lane_base + 32 * c_first, o[0]);
 #pragma unroll 1
@@ -783,20 +785,29 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
                   stg_256(orow + 32 * cc, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
                   stg_256(orow + 32 * cc + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
                 }
-              } else if (valid) {
+              } else {
+                // split unit: half precision with the chunk's power-of-two scale (see "Split partials")
+                float x[32], mx = 0.f;
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj)
-                  stg_256(prow + 32 * cc + 8 * jj,
-                          __float_as_uint(__uint_as_float(o[e][8 * jj + 0]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 1]) * inv),
-                          __float_as_uint(__uint_as_float(o[e][8 * jj + 2]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 3]) * inv),
-                          __float_as_uint(__uint_as_float(o[e][8 * jj + 4]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 5]) * inv),
-                          __float_as_uint(__uint_as_float(o[e][8 * jj + 6]) * inv), __float_as_uint(__uint_as_float(o[e][8 * jj + 7]) * inv));
+                for (int jj = 0; jj < 32; ++jj) { x[jj] = __uint_as_float(o[e][jj]) * inv; mx = fmaxf(mx, fabsf(x[jj])); }
+                float f;
+                const uint32_t sb = partial_scale_byte(mx, &f);
+                if (cq + e < 4) sc_lo |= sb << (8 * (cq + e)); else sc_hi |= sb << (8 * (cq + e - 4));
+                uint32_t w[16];
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) w[jj] = pack_f16x2(x[2 * jj] * f, x[2 * jj + 1] * f);
+                if (valid) {
+                  stg_256(hrow + 32 * cc, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                  stg_256(hrow + 32 * cc + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+                }
               }
             }
           }
+          if (valid && slot >= 0)
+            *reinterpret_cast<uint2*>(partial_scales(prm) + prow * 16 + c_first) = make_uint2(sc_lo, sc_hi);
           if (valid && !partner) {
             if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + row] = lse;
-            else prm.part_lse[static_cast<size_t>(slot) * kItemRows + half * kRowBlock + r] = lse;
+            else prm.part_lse[prow] = lse;
           }
           tc_fence_before_sync();
           if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 11 + 4 * un); };

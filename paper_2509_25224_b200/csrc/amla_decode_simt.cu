@@ -150,11 +150,22 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt_kernel(DecodeParams p
           }
           if (lane == 0) prm.lse[static_cast<size_t>(b) * prm.R + r0 + row] = lse;
         } else {
-          float* prow = prm.part_o + (static_cast<size_t>(slot) * kRowBlock + row) * kDv;
+          // half precision with one power-of-two scale per 32-column chunk (see "Split partials"): the 16 lanes of a
+          // half-warp hold one chunk of the row in every round
+          const size_t prow = static_cast<size_t>(slot) * kRowBlock + row;
+          uint32_t* hrow = reinterpret_cast<uint32_t*>(partial_halves(prm) + prow * kDv);
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            reinterpret_cast<float2*>(prow)[lane + 32 * i] = make_float2(O[rr][2 * i] * inv, O[rr][2 * i + 1] * inv);
-          if (lane == 0) prm.part_lse[static_cast<size_t>(slot) * kRowBlock + row] = lse;
+          for (int i = 0; i < 8; ++i) {
+            const float x0 = O[rr][2 * i] * inv, x1 = O[rr][2 * i + 1] * inv;
+            float mx = fmaxf(fabsf(x0), fabsf(x1));
+#pragma unroll
+            for (int o = 8; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float f;
+            const uint32_t sb = partial_scale_byte(mx, &f);
+            hrow[lane + 32 * i] = pack_f16x2(x0 * f, x1 * f);
+            if ((lane & 15) == 0) partial_scales(prm)[prow * 16 + 2 * i + (lane >> 4)] = static_cast<uint8_t>(sb);
+          }
+          if (lane == 0) prm.part_lse[prow] = lse;
         }
       }
     }

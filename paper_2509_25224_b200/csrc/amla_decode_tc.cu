@@ -814,7 +814,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
           const int rows_here = min(32, u.nrows - wid * 32);          // valid rows of this warp's 32 (may be <= 0)
           __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + u.r0 + wid * 32) * kDv;
-          float* pbase = prm.part_o + (static_cast<size_t>(slot < 0 ? 0 : slot) * kRowBlock + wid * 32) * kDv;
+          const size_t prow0 = static_cast<size_t>(slot < 0 ? 0 : slot) * kRowBlock + wid * 32;   // this warp's first row of the partial arrays
+          uint16_t* hbase = partial_halves(prm) + prow0 * kDv;
+          unsigned long long sc_lo = 0, sc_hi = 0;                    // this thread's row: sixteen scale bytes
           uint32_t o[2][32];
           tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
 #pragma unroll 1
@@ -844,26 +846,37 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                   if (row < rows_here) *reinterpret_cast<uint4*>(obase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * j) = v;
                 }
               } else {
+                // split unit: half precision with the chunk's power-of-two scale (see "Split partials")
+                float x[32], mx = 0.f;
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < 32; ++j) { x[j] = __uint_as_float(o[e][j]) * inv; mx = fmaxf(mx, fabsf(x[j])); }
+                float f;
+                const uint32_t sb = partial_scale_byte(mx, &f);
+                if (cc < 8) sc_lo |= static_cast<unsigned long long>(sb) << (8 * cc); else sc_hi |= static_cast<unsigned long long>(sb) << (8 * (cc - 8));
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
                   st_shared_v4(epi + lane * 128 + ((j ^ (lane & 7)) << 4),
-                               __float_as_uint(__uint_as_float(o[e][4 * j + 0]) * inv), __float_as_uint(__uint_as_float(o[e][4 * j + 1]) * inv),
-                               __float_as_uint(__uint_as_float(o[e][4 * j + 2]) * inv), __float_as_uint(__uint_as_float(o[e][4 * j + 3]) * inv));
+                               pack_f16x2(x[8 * j + 0] * f, x[8 * j + 1] * f), pack_f16x2(x[8 * j + 2] * f, x[8 * j + 3] * f),
+                               pack_f16x2(x[8 * j + 4] * f, x[8 * j + 5] * f), pack_f16x2(x[8 * j + 6] * f, x[8 * j + 7] * f));
                 __syncwarp();
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {                         // 4 rows x 128 B per instruction
-                  const int row = 4 * k + (lane >> 3), j = lane & 7;
+                for (int k = 0; k < 4; ++k) {                         // 8 rows x 64 B per instruction
+                  const int row = 8 * k + (lane >> 2), j = lane & 3;
                   uint4 v;
                   asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                                : "r"(epi + row * 128 + ((j ^ (row & 7)) << 4)));
-                  if (row < rows_here) *reinterpret_cast<uint4*>(pbase + static_cast<size_t>(row) * kDv + 32 * cc + 4 * j) = v;
+                  if (row < rows_here) *reinterpret_cast<uint4*>(hbase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * j) = v;
                 }
               }
             }
           }
           if (valid) {
-            if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
-            else prm.part_lse[static_cast<size_t>(slot) * kRowBlock + r] = lse;
+            if (slot < 0) {
+              prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
+            } else {
+              prm.part_lse[static_cast<size_t>(slot) * kRowBlock + r] = lse;
+              *reinterpret_cast<uint4*>(partial_scales(prm) + (static_cast<size_t>(slot) * kRowBlock + r) * 16) = make_uint4(static_cast<uint32_t>(sc_lo), static_cast<uint32_t>(sc_lo >> 32), static_cast<uint32_t>(sc_hi), static_cast<uint32_t>(sc_hi >> 32));
+            }
           }
           tc_fence_before_sync();
           if (tid == 0) AMLA_STAMP(prm, part, 19, un);

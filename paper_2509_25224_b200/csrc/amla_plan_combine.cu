@@ -89,21 +89,36 @@ __global__ void __launch_bounds__(128) combine_kernel(DecodeParams prm) {
   const int nsplit = info.y;
   if (nsplit == 1) return;
 
+  // a lane merges 16 consecutive columns (half of a 32-column chunk: one scale byte per split)
+  const uint16_t* halves = partial_halves(prm);
+  const uint8_t* scales = partial_scales(prm);
   float acc[16];
   float tot = 0.f, mx;
+  auto accumulate = [&](float w, uint32_t scale_byte, const uint4& a, const uint4& b) {
+    const float ws = w * partial_unscale(scale_byte);
+    const uint32_t h[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float2 v = unpack_f16x2(h[i]);
+      acc[2 * i] += ws * v.x;
+      acc[2 * i + 1] += ws * v.y;
+    }
+  };
   if (nsplit <= kFastSplits) {
     // everything is requested before anything is used
     float ls[kFastSplits];
-    float4 v[kFastSplits][4];
+    uint4 va[kFastSplits], vb[kFastSplits];
+    uint32_t sc[kFastSplits];
 #pragma unroll
     for (int s = 0; s < kFastSplits; ++s) {
       ls[s] = -INFINITY;
       if (s < nsplit) {
         const size_t prow = static_cast<size_t>(Plan::slot_of_split(info.x, s)) * prm.item_rows + rr;
         ls[s] = prm.part_lse[prow];
-        const float4* src = reinterpret_cast<const float4*>(prm.part_o + prow * kDv);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) v[s][i] = src[i * 32 + lane];
+        sc[s] = scales[prow * 16 + (lane >> 1)];
+        const uint4* src = reinterpret_cast<const uint4*>(halves + prow * kDv) + 2 * lane;
+        va[s] = src[0];
+        vb[s] = src[1];
       }
     }
     mx = ls[0];
@@ -117,11 +132,7 @@ __global__ void __launch_bounds__(128) combine_kernel(DecodeParams prm) {
       if (s < nsplit) {
         const float w = expf(ls[s] - mx);             // 0 for a split that saw nothing
         tot += w;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          acc[4 * i + 0] += w * v[s][i].x; acc[4 * i + 1] += w * v[s][i].y;
-          acc[4 * i + 2] += w * v[s][i].z; acc[4 * i + 3] += w * v[s][i].w;
-        }
+        accumulate(w, sc[s], va[s], vb[s]);
       }
     }
   } else {
@@ -150,26 +161,22 @@ __global__ void __launch_bounds__(128) combine_kernel(DecodeParams prm) {
         const float w = __shfl_sync(0xffffffffu, my_w, j);
         const int slot = __shfl_sync(0xffffffffu, my_slot, j);
         tot += w;
-        const float* src = prm.part_o + (static_cast<size_t>(slot) * prm.item_rows + rr) * kDv;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float4 x = *reinterpret_cast<const float4*>(src + i * 128 + lane * 4);
-          acc[4 * i + 0] += w * x.x; acc[4 * i + 1] += w * x.y;
-          acc[4 * i + 2] += w * x.z; acc[4 * i + 3] += w * x.w;
-        }
+        const size_t prow = static_cast<size_t>(slot) * prm.item_rows + rr;
+        const uint4* src = reinterpret_cast<const uint4*>(halves + prow * kDv) + 2 * lane;
+        accumulate(w, scales[prow * 16 + (lane >> 1)], src[0], src[1]);
       }
     }
   }
   const float inv = 1.f / tot;
+  uint32_t pk[8];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __nv_bfloat162 lo = __floats2bfloat162_rn(acc[4 * i + 0] * inv, acc[4 * i + 1] * inv);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(acc[4 * i + 2] * inv, acc[4 * i + 3] * inv);
-    uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(orow + i * 128 + lane * 4) = pk;
+  for (int i = 0; i < 8; ++i) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(acc[2 * i] * inv, acc[2 * i + 1] * inv);
+    pk[i] = *reinterpret_cast<uint32_t*>(&v);
   }
+  uint4* dst = reinterpret_cast<uint4*>(orow + 16 * lane);
+  dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+  dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
   if (lane == 0) *lrow = mx + logf(tot);
 #ifdef AMLA_TRACE
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));

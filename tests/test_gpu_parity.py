@@ -192,16 +192,27 @@ def test_rerun_is_bit_identical():
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
 
 
-def test_matches_algorithm2_simulator_closely():
-    # the CPU Algorithm-2 simulator uses the same readings; agreement should be far tighter than the
-    # oracle tolerance (both round P to bf16 and accumulate in fp32)
+def test_matches_algorithm2_simulator_closely(capsys):
+    # The CPU Algorithm-2 simulator uses the same readings; agreement should be far tighter than the oracle tolerance
+    # (both round P to bf16 and accumulate in fp32).  The sequence is split over many SM groups here, and the partial
+    # outputs travel in half precision (11 significant bits against the 8 of the bf16 result), so an element may land
+    # on the neighbouring bf16 value: at most one bf16 unit in the last place anywhere, most elements identical.
     w = synth.config_stress(B=1, N=2048)
     out, lse, _ = run_gpu(w, binding.RESCALE_ALG2)          # tau = 0, as the simulator
     kv = synth.bf16_bits_to_f32(synth.logical_kv_rows(w, 0))
     q = synth.bf16_bits_to_f32(w.q[0, 0])
     so, sl = S.amla(q, kv, kv[:, :512], w.scale, 64)
-    so = S.bf16_round(so)
-    assert np.abs(out[0, 0] - so).max() < 4e-3
+    so = S.bf16_round(so).astype(np.float64)
+    diff = np.abs(out[0, 0] - so)
+    big = np.maximum(np.abs(so), np.abs(out[0, 0]))
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(big, 2.0 ** -126))) - 7)      # bf16: 8 significant bits
+    same = float((diff == 0).mean())
+    with capsys.disabled():
+        print(f"\nvs Algorithm-2 simulator: identical {same:.3f}, max diff {diff.max():.3e}, mean diff {diff.mean():.2e}")
+    # one unit in the last place of the larger of the two, or (small elements of a row of large ones) the absolute
+    # bound this test had with FP32 partials
+    assert (diff <= np.maximum(ulp, 4e-3)).all()
+    assert same >= 0.9 and diff.mean() < 1e-4
     assert np.abs(lse[0, 0] - sl).max() < 1e-4
 
 
