@@ -6,10 +6,10 @@
 //       memory as the A operand, the 64 RoPE columns in shared memory.  K arrives by TMA in slots of
 //       128 keys x 192 columns (two pages stacked, one 4-D box each), three slots per score tile,
 //       through a ring; S = Q K^T (128 x 128, FP32) by tcgen05.mma into a double-buffered TMEM tile.  The
-//       two softmax warpgroups (two threads per query row, one per 64-key page of the tile) run
-//       Algorithm 2's per-row recurrence (lines 5-12) once per score tile and send the bf16
-//       probabilities P~ = bf16(P * S16) of their page plus the per-row integer N into the value CTA
-//       with asynchronous remote stores counted on a barrier there.
+//       softmax warpgroup runs Algorithm 2's per-row recurrence (lines 5-12) once per score tile,
+//       writes the bf16 probabilities P~ = bf16(P * S16) of each 64-key half plus the per-row integer
+//       N into a local staging buffer, and four copy warps move it into the value CTA with
+//       asynchronous remote stores counted on a barrier there.
 //   value CTA (cluster rank 1)   the whole FP32 accumulator O (128 x 512) lives in its tensor memory;
 //       V (first 512 columns of the same cache rows) arrives by TMA in slots of 64 keys x 256
 //       columns through a 4-slot ring; a correction warpgroup applies N to the bit patterns of O
@@ -34,10 +34,11 @@ using namespace sm100;
 
 namespace {
 
+constexpr int kNumCopyWarps = 4;         // score CTA: warps that move staged P~ to the value CTA
 #ifdef AMLA_TRACE
-constexpr int kThreads = 32 * 11;        // trace builds add a last warp, which watches the K slots fill
+constexpr int kThreads = 32 * (7 + kNumCopyWarps);   // trace builds add a last warp, which watches the K slots fill
 #else
-constexpr int kThreads = 32 * 10;        // warps 0-3 and 6-9: softmax (score CTA) / correction + epilogue (value CTA), 4: TMA producers, 5: MMA issuer + TMEM alloc
+constexpr int kThreads = 32 * (6 + kNumCopyWarps);   // warps 0-3: softmax / correction, 4: TMA producers, 5: MMA issuer + TMEM alloc, 6..: P copy
 #endif
 constexpr uint32_t kBoxBytes = 64 * 64 * 2;             // one 64-key x 64-column TMA box
 constexpr uint32_t kPBytes = 128 * 64 * 2;              // P~ of one 64-key half: 128 rows x 128 B
@@ -51,9 +52,8 @@ constexpr uint32_t kKPageBytes = 3 * kBoxBytes;         // 64 keys x 3 column bl
 constexpr uint32_t kKSlotBytes = 2 * kKPageBytes;       // 128 keys x 192 columns (two pages stacked)
 constexpr uint32_t kKGroupStride = 3 * 1024;            // distance between 8-row groups inside a slot
 constexpr uint32_t kOffQRope = 0;                       // 128 rows x 64 bf16, 128-byte swizzle
-constexpr uint32_t kOffXchg = 128 * 64 * 2;             // float [2 exchanges in flight][2 warpgroups][128 rows]: what the two threads of a row tell each other
-constexpr uint32_t kOffStage = kOffXchg + 2 * 1024;     // 8 softmax warps x 2 KB: half of a warp's 32 rows of P~ at a time, in the byte order of the P buffer
-constexpr uint32_t kOffK = kOffStage + 8 * 2048;
+constexpr uint32_t kOffStage = 128 * 64 * 2;            // kPStride: P~ and N of a page, before the copy warps move them to the value CTA
+constexpr uint32_t kOffK = kOffStage + kPStride;
 constexpr uint32_t kEndA = kOffK + kNumKSlots * kKSlotBytes;
 // ---- value CTA
 constexpr int kNumVSlots = 4;
@@ -65,10 +65,10 @@ constexpr uint32_t kOffEpi = kOffFin + 2 * 128 * 8;     // epilogue transpose ti
 constexpr uint32_t kEndB = kOffEpi + 4 * 32 * 128;
 // ---- both: the barriers sit at the same offset, so that one multicast commit can reach the two CTAs
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
-constexpr uint32_t kBarBytes = 256;
+constexpr uint32_t kBarBytes = 512;
 // ---- both: a copy of the schedule prefix and of the sequence lengths for batches of up to kSmemPlanItems items,
 // so that the roles' schedule look-ups (a dozen dependent loads per unit) stay on chip
-constexpr int kSmemPlanItems = 64;
+constexpr int kSmemPlanItems = 128;
 constexpr uint32_t kOffPlan = kOffBars + kBarBytes;                          // int [kSmemPlanItems + 1] prefix
 constexpr uint32_t kOffSeqlens = kOffPlan + ((kSmemPlanItems + 1) * 4 + 15) / 16 * 16;   // int [kSmemPlanItems] sequence lengths
 constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
@@ -85,7 +85,7 @@ constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 column
 // score CTA the same arrival (multicast commit) frees the page's P buffer for the softmax (PEMPTY).
 enum { X_PV = 0, X_COMMON = X_PV + kNumP };
 enum { A_KFULL = X_COMMON, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2,
-       A_XCHG = A_SEMPTY + 2, A_QREADY = A_XCHG + 4, A_QFREE, A_FINFREE, A_NUM = A_FINFREE + 2 };
+       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2, A_QFREE, A_FINFREE, A_NUM = A_FINFREE + 2 };
 enum { B_VFULL = X_COMMON, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP,
        B_FINFULL = B_OREADY + kNumP, B_NUM = B_FINFULL + 2 };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
@@ -200,76 +200,49 @@ struct RoleCtx {
   int part, tid;
 };
 
-// One arrival per warp on a barrier of this CTA, after every lane's preceding work.
-__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
-  __syncwarp();
-  if (lane == 0) mbar_arrive(bar);
-}
-
-// One softmax warp's work on one unit.  Two threads share a query row: the thread of warpgroup A (warps 0-3) takes
-// the first 64-key page of every score tile, the thread of warpgroup B (warps 6-9, which reach the same
-// tensor-memory lanes as warps 2, 3, 0, 1) the second (a unit's last tile may have one page only; B then sits the
-// tile out).  Each reads its 64 scores into registers (the score tile is free for the next QK^T from then on), the two
-// exchange their maxima through shared memory and run Algorithm 2's per-row recurrence (lines 5-12) on the same
-// inputs, so both hold the same state; the row sum of line 6 is kept as two partial sums that meet at the end of
-// the unit.  P~ = bf16(P * S16) and the row's integer N (first page only: the second leaves O alone) go into a P
-// buffer of the value CTA by asynchronous remote stores counted on its barrier; the final scalars 1/(l*S16) and lse
-// (line 20) follow at the end of the unit.  Returns (pages so far) << 32 | (score tiles so far) << 1 | ok.
+// The softmax warpgroup's work on one unit: its score tiles, then the final scalars for the value CTA.  A function
+// of its own, so that it can also be run and timed outside the kernel.  Returns
+// (pages so far) << 32 | (score tiles so far) << 1 | ok.
 template <int kMode>
 __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const RoleCtx c, const Unit u, uint32_t un, uint32_t gt, uint32_t gs) {
-  const int tid = c.tid, wid = tid >> 5, lane = tid & 31, part = c.part;
+  const int tid = c.tid, wid = tid >> 5, part = c.part;
   const uint32_t smem_base = c.smem_base, bars = c.bars, tbase = c.tbase, peerB_bars = c.peerB_bars, peerB_base = c.peerB_base;
   auto bar = [&](int i) { return bars + 8u * i; };
   (void)part;
   bool ok = true;
-  const int hsel = wid >= 6 ? 1 : 0;                   // which page of every tile
-  const int quarter = wid & 3;                         // tensor-memory lane quarter of this warp
-  const int r = quarter * 32 + lane;                   // query row
-  const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+  const int r = tid;
+  const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
   const bool scale_nonneg = prm.scale_log2 >= 0.f;
   const uint32_t mask_fill = __float_as_uint(scale_nonneg ? -INFINITY : INFINITY);
-  RowState st;
-  row_state_init(st);
-  const int tok = (u.r0 + r) / prm.H;
-  const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);          // keys 0..visible-1 are seen by this row
-  const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // pages from here on may hold hidden keys
-  uint32_t xc = gs + un;                                // exchanges so far: one per tile, one at the end of a unit
-  const uint32_t xbar = bar(A_XCHG + quarter);
-  // tells the row's other thread `mine`, returns what it told
-  auto exchange = [&](float mine) -> float {
-    const uint32_t slot = smem_base + kOffXchg + (xc & 1) * 1024;
-    st_shared_b32(slot + (hsel * 128 + r) * 4, __float_as_uint(mine));
-    warp_arrive(xbar, lane);
-    ok = warp_wait(xbar, xc & 1);
-    ++xc;
-    return __uint_as_float(ld_shared_b32(slot + ((hsel ^ 1) * 128 + r) * 4));
-  };
+  {
+    RowState st;
+    row_state_init(st);
+    const int tok = (u.r0 + r) / prm.H;
+    const int visible = min(u.n_b, u.n_b - prm.Sq + tok + 1);          // keys 0..visible-1 are seen by this row
+    const int first_masked_tile = max(u.n_b - prm.Sq + 1, 0) / kPage;  // pages from here on may hold hidden keys
 
-  for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
-    const int npages = min(2, u.t1 - t);
-    const bool have_page = hsel < npages;               // B has nothing to do in a one-page tile
-    const uint32_t sb = gs & 1;
-    ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
-    if (!ok) break;
-    tc_fence_after_sync();
-    if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
-    const uint32_t scol = tbase + lane_base + kSCol + 128 * sb + 64 * hsel;
-    const int nvis = visible - (t + hsel) * kPage;       // keys of this page the row sees (may be <= 0)
-    uint32_t b0[32], b1[32];
-    if (have_page) {
-      tmem_ld_32x32b_x32(scol, b0);
-      tmem_ld_32x32b_x32(scol + 32, b1);
-      tmem_wait_ld();
-    }
-    tc_fence_before_sync();
-    warp_arrive(bar(A_SEMPTY + sb), lane);               // the scores are in registers
-    if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
-    auto tile_body = [&](auto general_c) {
+    for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
+      const int npages = min(2, u.t1 - t);
+      const uint32_t sb = gs & 1;
+      ok = warp_wait(bar(A_SFULL + sb), (gs >> 1) & 1);
+      if (!ok) break;
+      tc_fence_after_sync();
+      if (tid == 0) AMLA_STAMP(prm, part, 5, gt);
+      const uint32_t scol = tbase + lane_base + kSCol + 128 * sb;
+      const int nvis = visible - t * kPage;              // keys of this score tile the row sees (may be <= 0)
+      // Two compilations of the tile: the plain one (every key visible, non-negative scale), and the general one
+      // with the visibility masks and the sign of the scale; a run-time flag inside one body costs the plain
+      // tiles their instruction schedule.
+      auto tile_body = [&](auto general_c) {
       constexpr bool kGeneral = decltype(general_c)::value;
       constexpr bool masked = kGeneral;
       const bool scale_nn = kGeneral ? scale_nonneg : true;
-      // lines 5-6: running max on the raw scores (the scale is folded into the FMA below)
-      float ext = scale_nn ? -INFINITY : INFINITY, ext_b = ext;
+
+      // The S tile is read from tensor memory in 32-column chunks, twice (maximum, then exponentials); the load
+      // of the next chunk is always in flight while a chunk is processed, so that the TMEM latency is hidden.
+      uint32_t b0[32], b1[32];
+      // lines 5-6: running max, taken on the raw scores (the scale is folded into the FMA below)
+      float ext = scale_nn ? -INFINITY : INFINITY, ext_b = ext;      // two chains: half the dependent latency
       auto chunk_max = [&](uint32_t (&v)[32], int col0) {
         if (masked) {
 #pragma unroll
@@ -289,23 +262,28 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           }
         }
       };
-      if (have_page) {
-        chunk_max(b0, 0);
-        chunk_max(b1, 32);
+      tmem_ld_32x32b_x32(scol, b0);
+#pragma unroll 1
+      for (int h = 0; h < npages; ++h) {
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+        chunk_max(b0, 64 * h);
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + (h + 1 < npages ? 64 * (h + 1) : 0), b0);   // next half, or the first chunk again for the second pass
+        chunk_max(b1, 64 * h + 32);
       }
       ext = scale_nn ? fmaxf(ext, ext_b) : fminf(ext, ext_b);
-      const float mine = (have_page && nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
-      const float tmax = fmaxf(mine, exchange(mine));
-      if (!ok) return;
+      const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
       const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
-      if (!have_page) { st.l *= sp.l_up; return; }
-      // Line 10's factor S16 goes into the exponential's argument (the remark after Algorithm 2).  The row sum of
-      // line 6 is the sum of the same FP32 values, taken before the bf16 cast and divided by S16 once per tile.
+      // Line 10's factor S16 goes into the exponential's argument (the paper's remark after Algorithm 2):
+      // P * S16 = 2^(a - m + log2 S16).  The row sum of line 6 is the sum of the same FP32 values, taken
+      // before the bf16 cast and divided by S16 once per tile.
       const float nsub = log2f_approx(sp.p_scale) - sp.m2_sub;
       float rs0 = 0.f, rs1 = 0.f;
       const uint64_t sc2 = pack_f32x2(prm.scale_log2, prm.scale_log2), ns2 = pack_f32x2(nsub, nsub);
       uint64_t rsa = pack_f32x2(0.f, 0.f), rsb = rsa;
       uint32_t pk[32];
+      // lines 6, 10 for 32 columns: P, row sum (FP32, unscaled), P~ = bf16(P * S16), two elements per instruction
       auto chunk_exp = [&](const uint32_t (&v)[32], int col0, int k0) {
         if (masked) {
 #pragma unroll
@@ -329,69 +307,65 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
           }
         }
       };
-      chunk_exp(b0, 0, 0);
-      chunk_exp(b1, 32, 16);
+#pragma unroll 1
+      for (int h = 0; h < npages; ++h) {
+        tmem_wait_ld();
+        tmem_ld_32x32b_x32(scol + 64 * h + 32, b1);
+        chunk_exp(b0, 64 * h, 0);
+        tmem_wait_ld();
+        if (h + 1 < npages) {
+          tmem_ld_32x32b_x32(scol + 64 * (h + 1), b0);
+        } else {                       // the score tile has been read for the last time
+          tc_fence_before_sync();
+          mbar_arrive(bar(A_SEMPTY + sb));
+          if (tid == 0) AMLA_STAMP2(prm, part, 6, gt);
+        }
+        // One staging buffer: the copy warps of the previous page must have read it into registers.  The barrier is
+        // probed here, ahead of the last chunk's arithmetic, so that the probe's latency is not exposed (this warp
+        // is alone on its scheduler); the blocking wait runs only if the probe came too early.
+        const bool stage_free = gt == 0 || mbar_probe(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+        chunk_exp(b1, 64 * h + 32, 16);
+        // stage P~ and N; the copy warps ship them to the value CTA
+        const uint32_t s2 = gt & 1;
+        if (tid == 0) AMLA_STAMP2(prm, part, 7, gt);
+        if (!__all_sync(0xffffffffu, stage_free)) ok = warp_wait(bar(A_STAGEFREE + ((gt - 1) & 1)), ((gt - 1) >> 1) & 1);
+        if (!ok) break;
+        if (tid == 0) AMLA_STAMP2(prm, part, 8, gt);
+        const uint32_t stg = smem_base + kOffStage;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          st_shared_v4(stg + sw128_offset(r, c), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        // the rescale (if any) belongs to the first half; the second half leaves O alone
+        const uint32_t nword = (kMode == 2) ? __float_as_uint(h == 0 ? sp.l_up : 1.f)
+                                            : static_cast<uint32_t>(h == 0 ? sp.n_bits : 0);
+        st_shared_b32(stg + kPBytes + r * 4, nword);
+        mbar_arrive(bar(A_PSTAGED + s2));
+        if (tid == 0) AMLA_STAMP(prm, part, 9, gt);
+        ++gt;
+      }
       {
         float s0, s1;
         unpack_f32x2(add_f32x2(rsa, rsb), s0, s1);
-        st.l = st.l * sp.l_up + __fdividef((rs0 + s0) + (rs1 + s1), sp.p_scale);   // this thread's share of the row sum
+        rs0 += s0; rs1 += s1;
       }
-      // ---- ship the page.  A thread's 128 bytes are eight 16-byte pieces of one row; sent as they are, every store
-      // instruction of the warp would be 32 separate small remote writes.  The warp's 32 rows are a contiguous 4 KB
-      // block of the P buffer, so they pass, 16 rows at a time, through a 2 KB staging block of the warp's own and
-      // leave in instructions that cover 512 contiguous bytes each.
-      const uint32_t gp = gt + hsel;                          // page number within the cluster's work
-      const uint32_t pb = gp % kNumP;
-      ok = warp_wait(bar(X_PV + pb), ((gp / kNumP) & 1) ^ 1);      // the P V that last read the buffer is done
-      if (!ok) return;
-      const uint32_t pfull = peerB_bars + 8u * (B_PFULL + pb);
-      const uint32_t dstp = peerB_base + kOffP + pb * kPStride;
-      if (quarter == 0 && lane == 0) { AMLA_STAMP2(prm, part, 23, gp); mbar_arrive_expect_tx_cluster(pfull, kPXfer); }
-      const uint32_t stage = smem_base + kOffStage + (hsel * 4 + quarter) * 2048;
-#pragma unroll
-      for (int h2 = 0; h2 < 2; ++h2) {
-        if ((lane >> 4) == h2) {
-#pragma unroll
-          for (int cc = 0; cc < 8; ++cc)
-            st_shared_v4(stage + sw128_offset(lane & 15, cc), pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
-        }
-        __syncwarp();
-        uint32_t v[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i][0]), "=r"(v[i][1]), "=r"(v[i][2]), "=r"(v[i][3])
-                       : "r"(stage + i * 512 + lane * 16));
-        __syncwarp();
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          st_async_v4(dstp + quarter * 4096 + h2 * 2048 + i * 512 + lane * 16, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
-      }
-      const uint32_t nword = (kMode == 2) ? __float_as_uint(hsel == 0 ? sp.l_up : 1.f)
-                                          : static_cast<uint32_t>(hsel == 0 ? sp.n_bits : 0);
-      st_async_b32(dstp + kPBytes + r * 4, nword, pfull);
-      if (tid == 0) AMLA_STAMP(prm, part, 9, gp);
-    };
-    if (t + npages > first_masked_tile || !scale_nonneg) tile_body(std::true_type{});
-    else tile_body(std::false_type{});
-    gt += npages;
-  }
-  // line 20 scalars: 1 / (l * S16) and lse = m + ln l, from both threads' shares of the row sum; B sends them
-  if (ok) {
-    const float l_all = st.l + exchange(st.l);
-    if (ok && hsel == 1) {
-      // The two-entry buffer of the value CTA is written for unit `un` only after the epilogue of unit un - 2 has read
-      // its entry (nothing else keeps the softmax from running two short units ahead of the epilogue).
-      ok = warp_wait<true>(bar(A_FINFREE + (un & 1)), ((un >> 1) & 1) ^ 1);
-      if (ok) {
-        const bool live = l_all > 0.f;
-        const float inv = live ? prm.out_scale / (l_all * st.s_out) : 0.f;
-        const float lse = live ? (st.m2 + log2f(l_all)) * kLn2 : -INFINITY;
-        // asynchronous remote stores counted on the barrier: no thread has to wait for a cluster-scope release
-        const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;
-        const uint32_t fbar = peerB_bars + 8u * (B_FINFULL + (un & 1));
-        if (wid == 6 && lane == 0) mbar_arrive_expect_tx_cluster(fbar, 128 * 8);
-        st_async_v2(fdst, __float_as_uint(inv), __float_as_uint(lse), fbar);
-      }
+      st.l = st.l * sp.l_up + __fdividef(rs0 + rs1, sp.p_scale);
+      };
+      if (t + npages > first_masked_tile || !scale_nonneg) tile_body(std::true_type{});
+      else tile_body(std::false_type{});
+    }
+    // line 20 scalars: 1 / (l * S16) and lse = m + ln l
+    // The two-entry buffer of the value CTA is written for unit `un` only after the epilogue of unit un - 2 has read
+    // its entry (nothing else keeps this warpgroup from running two short units ahead of the epilogue).
+    if (ok) ok = warp_wait<true>(bar(A_FINFREE + (un & 1)), ((un >> 1) & 1) ^ 1);
+    if (ok) {
+      const bool live = st.l > 0.f;
+      const float inv = live ? prm.out_scale / (st.l * st.s_out) : 0.f;
+      const float lse = live ? (st.m2 + log2f(st.l)) * kLn2 : -INFINITY;
+      // asynchronous remote stores counted on the barrier: no thread has to wait for a cluster-scope release
+      const uint32_t fdst = peerB_base + kOffFin + ((un & 1) * 128 + r) * 8;
+      const uint32_t fbar = peerB_bars + 8u * (B_FINFULL + (un & 1));
+      if (tid == 0) mbar_arrive_expect_tx_cluster(fbar, 128 * 8);
+      st_async_v2(fdst, __float_as_uint(inv), __float_as_uint(lse), fbar);
     }
   }
   return (static_cast<uint64_t>(gt) << 32) | (static_cast<uint64_t>(gs) << 1) | (ok ? 1u : 0u);
@@ -426,9 +400,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     if (is_score) {
       for (int i = 0; i < kNumKSlots; ++i) { mbar_init(bar(A_KFULL + i), 1); mbar_init(bar(A_KEMPTY + i), 1); }
       for (int i = 0; i < 2; ++i) {
-        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 8);      // the eight softmax warps
+        mbar_init(bar(A_SFULL + i), 1); mbar_init(bar(A_SEMPTY + i), 128);
+        mbar_init(bar(A_PSTAGED + i), 128); mbar_init(bar(A_STAGEFREE + i), 2);
       }
-      for (int i = 0; i < 4; ++i) mbar_init(bar(A_XCHG + i), 2);                // the two warps that share 32 rows
       mbar_init(bar(A_QREADY), 256);
       mbar_init(bar(A_QFREE), 1);
       for (int i = 0; i < 2; ++i) mbar_init(bar(A_FINFREE + i), 4);   // the four epilogue warps of the value CTA
@@ -509,12 +483,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     // ======================================================================= score CTA
     uint32_t gs = 0;    // score tiles (one or two pages) so far
     uint32_t gc = 0;    // K ring slots so far
-    if (wid < 4 || (wid >= 6 && wid < 10)) {
-      // ---- softmax warps: A = warps 0-3 (first page of every tile), B = warps 6-9 (second page).  At the start of
-      // a unit they bring in its Q rows: A the first 256 latent columns, B the other 256 and the RoPE columns.
-      const bool grp_b = wid >= 6;
-      const int qr = (wid & 3) * 32 + lane;
-      const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+    if (wid < 4) {
+      // ---- softmax warpgroup: thread = query row
+      const int r = tid;
+      const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
       const RoleCtx ctx{smem_base, bars, tbase, peerB_bars, peerB_base, prefix, seqlens, part, tid};
       while (ok && iter.next(u)) {
         // Q row -> tensor memory / shared memory (the previous unit's QK^T must be finished with it)
@@ -523,27 +495,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         tc_fence_after_sync();
         if (tid == 0) AMLA_STAMP(prm, part, 10, un);
         {
-          const bool valid = qr < u.nrows;
-          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? qr : 0)) * kDqk);
-          load_q_latent(qrow, valid, grp_b ? 4 : 0, tbase + q_lane_base + kQCol);
-          if (grp_b) {
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-              const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
-              st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
-            }
-          }
+          // this warpgroup brings in the first 256 latent columns of its rows; the copy warps, idle at this
+          // point, bring in the other 256 and the RoPE columns
+          const bool valid = r < u.nrows;
+          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDqk);
+          load_q_latent(qrow, valid, 0, tbase + lane_base + kQCol);
           tmem_wait_st();
-          if (grp_b) fence_proxy_async_smem();
         }
         tc_fence_before_sync();
         mbar_arrive(bar(A_QREADY));
         if (tid == 0) AMLA_STAMP(prm, part, 11, un);
-        if (grp_b) {                               // the next unit's Q goes to L2 while this one is computed
-          UnitIter peek = iter;
-          Unit nu;
-          if (peek.next(nu)) prefetch_q_row(prm, nu, qr);
-        }
         // the unit's score tiles and its final scalars
         const uint64_t ret = softmax_unit<kMode>(prm, ctx, u, un, gt, gs);
         gt = static_cast<uint32_t>(ret >> 32);
@@ -551,7 +512,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         ok = (ret & 1u) != 0;
         ++un;
       }
-      if (!ok && lane == 0) report_timeout(prm.status);
+      if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
       // ---- TMA producers: K, three slots (192 columns each) per score tile.  Lane l owns ring slot l and
       // loads every kNumKSlots-th slot of the sequence; the lanes poll without blocking, so that a slot that
@@ -671,7 +632,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         if (!ok) report_timeout(prm.status);
       }
 #ifdef AMLA_TRACE
-    } else if (wid == 10) {
+    } else if (wid == 6 + kNumCopyWarps) {
       // trace builds: lane l watches K slot l and stamps the arrival of its data (non-blocking polls)
       if (prm.trace) {
         Cursor<true> cur(prm, prefix, seqlens, part);
@@ -692,6 +653,67 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         }
       }
 #endif
+    } else if (wid >= 6 && wid < 6 + kNumCopyWarps) {
+      // ---- copy warps: staged P~ / N of a page -> a free P buffer of the value CTA, by asynchronous remote stores
+      // counted on its PFULL barrier.  (A bulk copy would queue behind the K loads in this SM's copy engine and
+      // arrive thousands of cycles later; remote stores issued by the softmax threads themselves would stall them
+      // at the rate of the SM-to-SM path.)  Warps c and c + 2 serve the pages of parity c -- staging buffer c --
+      // and move one half of the buffer each, so every warp sees every phase of the barriers it waits on.  The
+      // staging buffer is free as soon as both have read their half into registers.
+      {
+        const uint32_t c = (wid - 6) & 1, half = (wid - 6) >> 1;
+        constexpr int kChunks = 17;                         // 512-byte chunks per warp (33 in total)
+        const int qr = (wid & 3) * 32 + lane;               // query row whose second half this thread loads
+        const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+        while (ok && iter.next(u)) {
+          {
+            ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool valid = qr < u.nrows;
+            const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? qr : 0)) * kDqk);
+            load_q_latent(qrow, valid, 4, tbase + q_lane_base + kQCol);
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+              const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
+              st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
+            }
+            tmem_wait_st();
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(bar(A_QREADY));
+            ++un;
+            UnitIter peek = iter;              // the next unit's Q goes to L2 while this one is computed
+            Unit nu;
+            if (peek.next(nu)) prefetch_q_row(prm, nu, qr);
+          }
+          for (int t = u.t0; t < u.t1; ++t, ++gt) {
+            if ((gt & 1) != c) continue;
+            const uint32_t pb = gt % kNumP;
+            ok = warp_wait(bar(A_PSTAGED + c), (gt >> 1) & 1);
+            if (!ok) break;
+            const uint32_t src = smem_base + kOffStage + (half * kChunks * 32 + lane) * 16;
+            uint32_t v[kChunks][4];
+#pragma unroll
+            for (int i = 0; i < kChunks; ++i) {
+              if (half * kChunks + i < 33)
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i][0]), "=r"(v[i][1]), "=r"(v[i][2]), "=r"(v[i][3]) : "r"(src + i * 512));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(A_STAGEFREE + c));
+            ok = warp_wait(bar(X_PV + pb), ((gt / kNumP) & 1) ^ 1);      // P V that last read the buffer is done
+            if (!ok) break;
+            const uint32_t pfull = peerB_bars + 8u * (B_PFULL + pb);
+            const uint32_t dst = peerB_base + kOffP + pb * kPStride + (half * kChunks * 32 + lane) * 16;
+            if (lane == 0 && half == 0) { AMLA_STAMP2(prm, part, 23, gt); mbar_arrive_expect_tx_cluster(pfull, kPXfer); }
+#pragma unroll
+            for (int i = 0; i < kChunks; ++i) {
+              if (half * kChunks + i < 33) st_async_v4(dst + i * 512, v[i][0], v[i][1], v[i][2], v[i][3], pfull);
+            }
+          }
+        }
+        if (!ok && lane == 0) report_timeout(prm.status);
+      }
     }
   } else {
     // ======================================================================= value CTA
