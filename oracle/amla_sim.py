@@ -1,7 +1,7 @@
 """TEST INFRASTRUCTURE -- not part of the product path.
 
-CPU simulators, in numpy, of the two recurrences the paper states, written in
-the paper's order and notation so they can be checked against it by eye:
+CPU simulators, in numpy, of the two recurrences the paper states, in the
+paper's notation so they can be checked against it by eye:
 
 * ``flash_attention``  -- Algorithm 1 (tiled online softmax, "Base").
 * ``amla``             -- Algorithm 2 (AMLA): power-of-two reference n_i,
@@ -95,64 +95,80 @@ def flash_attention(Q, K, V, scale, tile, dtype=np.float64, low_precision_matmul
 
 def amla(Q, K, V, scale, tile, c_mode="appendix", skip_unchanged=True, guard=True,
          clamp=-30.0, tiny=1e-6, visible=None, trace=None):
-    """Algorithm 2 in FP32 with bf16 P (the mixed precision of Appendix A).
+    """AMLA (Algorithm 2; Eq. 3, Lemma 3.1, Appendix A) in FP32 with bf16 P, organised around its quantities.
 
-    Returns (O [G,Dv] float32, lse [G] float32).  ``trace``, if a list, receives one
-    dict per tile with the per-row scalars (m, n, S32, S16, c, eps, N).
+    Everything the rescaling needs depends on the running row maxima alone, so it is computed first, for all
+    tiles at once: the power-of-two reference n_i = round(-m_i / ln 2) (Eq. 3), S32_i = 1/r_i = exp(n_i ln 2 + m_i)
+    in [1/sqrt 2, sqrt 2], its bf16 rounding S16_i, the compensation c_i of Appendix A, the residual
+    eps_i = 1.5 (c_i / c_{i-1} - 1), and from them the integer N_i that Lemma 3.1 adds to the bit pattern of the
+    accumulator, (max(n_i - n_{i-1}, clamp) + eps_i + tiny) * 2^23 rounded.  The second part walks the tiles: P and the
+    row sum against the reference, P~ = bf16(P * S16_i), the integer add on O, O += P~ V.  The result is
+    O / (l * S16) of the last tile.
+
+    Returns (O [G,Dv] float32, lse [G] float32).  ``trace``, if a list, receives one dict per tile with the per-row
+    scalars (m, n, S32, S16, c, eps, N).
     """
     f = np.float32
     Q = np.asarray(Q, dtype=f); K = np.asarray(K, dtype=f); V = np.asarray(V, dtype=f)
     G, S2 = Q.shape[0], K.shape[0]
-    O = np.zeros((G, V.shape[1]), dtype=f)
-    m = np.full(G, -np.inf, dtype=f)
-    l = np.zeros(G, dtype=f)
-    n_prev = np.zeros(G, dtype=f)
-    c_prev = np.ones(G, dtype=f)
-    S16 = np.ones(G, dtype=f)
-    started = np.zeros(G, dtype=bool)       # row has received at least one P V product ("i > 1" per row)
-    for lo in range(0, S2, tile):
-        hi = min(S2, lo + tile)
-        S = (Q @ K[lo:hi].T).astype(f) * f(scale)                          # lines 4-5
+    bounds = [(lo, min(S2, lo + tile)) for lo in range(0, S2, tile)]
+    T = len(bounds)
+    if T == 0:
+        return np.zeros((G, V.shape[1]), dtype=f), np.full(G, -np.inf, dtype=f)
+
+    # ---- scores of every tile and the running maxima
+    tiles = []
+    for lo, hi in bounds:
+        S = (Q @ K[lo:hi].T).astype(f) * f(scale)
         if visible is not None:
             S = np.where(np.arange(lo, hi)[None, :] < np.asarray(visible)[:, None], S, f(-np.inf)).astype(f)
-        m_new = np.maximum(m, S.max(axis=1)).astype(f)
-        live = ~np.isneginf(m_new)
-        m_safe = np.where(live, m_new, f(0)).astype(f)
-        M_up = np.where(np.isneginf(m), f(0), np.exp((m - m_safe).astype(f))).astype(f)
-        n_i = np.rint(-m_safe / LN2).astype(f)                              # line 6
-        P = np.exp((S - m_safe[:, None]).astype(f)).astype(f)
-        l = (l * M_up + P.sum(axis=1, dtype=f)).astype(f)
-        S32 = np.exp((LN2 * (n_i + m_safe / LN2)).astype(f)).astype(f)      # line 7: 1/r_i
-        S16 = bf16_round(S32)                                               # line 8: 1/r'_i
-        if c_mode == "appendix":
-            c_i = (S16 / S32).astype(f)                                     # r_i / r'_i
-        elif c_mode == "listing":
-            c_i = (S32 / S16).astype(f)
-        elif c_mode == "none":
-            c_i = np.ones(G, dtype=f)
-        else:
-            raise ValueError(c_mode)
-        eps = (f(1.5) * (c_i / c_prev - f(1))).astype(f)                    # line 9
-        Pt = bf16_round((P * S16[:, None]).astype(f))                       # line 10
-        Nf = np.maximum(n_i - n_prev, f(clamp)).astype(np.float64)          # line 11 (exact in fp64)
-        N = np.rint((Nf + eps.astype(np.float64) + tiny) * 2.0 ** 23).astype(np.int64)   # line 12
-        changed = m_new != m
-        apply = started & live & (changed if skip_unchanged else True)
-        N = np.where(apply, N, 0)
-        O = exponent_add(O, N[:, None], guard=guard)                        # lines 13-16
-        O = (O + (Pt @ V[lo:hi]).astype(f)).astype(f)                       # lines 17-18
+        tiles.append(S)
+    m = np.maximum.accumulate(np.stack([S.max(axis=1) for S in tiles]).astype(f), axis=0)      # [T, G]
+    m_before = np.concatenate([np.full((1, G), -np.inf, dtype=f), m[:-1]])
+    live = ~np.isneginf(m)                                   # the row has seen a key by tile i
+    started = ~np.isneginf(m_before)                         # ... before tile i: O holds something to rescale
+    m_safe = np.where(live, m, f(0)).astype(f)
+
+    # ---- what the rescaling needs, for all tiles (Eq. 3, Appendix A)
+    n = np.rint(-m_safe / LN2).astype(f)
+    S32 = np.exp((LN2 * (n + m_safe / LN2)).astype(f)).astype(f)
+    S16 = bf16_round(S32)
+    if c_mode == "appendix":
+        c = (S16 / S32).astype(f)                            # r_i / r'_i
+    elif c_mode == "listing":
+        c = (S32 / S16).astype(f)
+    elif c_mode == "none":
+        c = np.ones((T, G), dtype=f)
+    else:
+        raise ValueError(c_mode)
+    # the scalars of the previous tile that had seen a key (n = 0, c = 1 before there is one)
+    n_before = np.concatenate([np.zeros((1, G), dtype=f), n[:-1]])
+    c_before = np.concatenate([np.ones((1, G), dtype=f), c[:-1]])
+    n_before = np.where(started, n_before, f(0)).astype(f)
+    c_before = np.where(started, c_before, f(1)).astype(f)
+    eps = (f(1.5) * (c / c_before - f(1))).astype(f)
+    dn = np.maximum(n - n_before, f(clamp)).astype(np.float64)
+    N = np.rint((dn + eps.astype(np.float64) + tiny) * 2.0 ** 23).astype(np.int64)
+    moved = (m != m_before) if skip_unchanged else np.ones((T, G), dtype=bool)
+    N = np.where(started & live & moved, N, 0)
+    l_up = np.where(started, np.exp((m_before - m_safe).astype(f)), f(0)).astype(f)       # exp(m_{i-1} - m_i)
+
+    # ---- the tiles: row sum, P~, integer add on O, accumulation
+    O = np.zeros((G, V.shape[1]), dtype=f)
+    l = np.zeros(G, dtype=f)
+    for i, (lo, hi) in enumerate(bounds):
+        P = np.exp((tiles[i] - m_safe[i][:, None]).astype(f)).astype(f)
+        l = (l * l_up[i] + P.sum(axis=1, dtype=f)).astype(f)
+        Pt = bf16_round((P * S16[i][:, None]).astype(f))
+        O = exponent_add(O, N[i][:, None], guard=guard)
+        O = (O + (Pt @ V[lo:hi]).astype(f)).astype(f)
         if trace is not None:
-            trace.append(dict(m=m_new.copy(), n=n_i.copy(), S32=S32.copy(), S16=S16.copy(),
-                              c=c_i.copy(), eps=eps.copy(), N=N.copy()))
-        upd = live
-        n_prev = np.where(upd, n_i, n_prev).astype(f)
-        c_prev = np.where(upd, c_i, c_prev).astype(f)
-        started = started | live
-        m = m_new
+            trace.append(dict(m=m[i].copy(), n=n[i].copy(), S32=S32[i].copy(), S16=S16[i].copy(),
+                              c=c[i].copy(), eps=eps[i].copy(), N=N[i].copy()))
     with np.errstate(divide="ignore", invalid="ignore"):
-        den = (l * S16).astype(f)
-        out = np.where(l[:, None] > 0, O / np.where(l > 0, den, f(1))[:, None], f(0)).astype(f)   # line 20
-        lse = np.where(l > 0, m + np.log(np.where(l > 0, l, f(1))), f(-np.inf)).astype(f)
+        den = (l * S16[-1]).astype(f)
+        out = np.where(l[:, None] > 0, O / np.where(l > 0, den, f(1))[:, None], f(0)).astype(f)
+        lse = np.where(l > 0, m[-1] + np.log(np.where(l > 0, l, f(1))), f(-np.inf)).astype(f)
     return out, lse
 
 
