@@ -300,7 +300,12 @@ __device__ __noinline__ uint32_t softmax_unit(const DecodeParams prm, const Role
       const float mine = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
       const float tmax = fmaxf(mine, exchange(mine));
       if (!ok) return;
-      const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
+      // Lazy reference: a row must move when its maximum exceeds the reference by more than tau.  The correction warp
+      // that serves these 32 rows pays for a rescale as soon as one of them moves, so when one must, every row of the
+      // warp whose maximum rose moves with it (moving early is always allowed: tau = 0 moves at every rise); the rows
+      // then tend to stay in step and the warp rescales on far fewer tiles.
+      const bool must = tmax > st.m2 + prm.tau;
+      const RowStep sp = row_step<kMode>(st, tmax, __any_sync(0xffffffffu, must) ? 0.f : prm.tau);
       if (tid == 0) QSTAMP(c.smem_base, 13, gs);
       // Line 10's factor S16 goes into the exponential's argument (the remark after Algorithm 2).  The row sum of
       // line 6 is the sum of the same FP32 values, taken before the bf16 cast and divided by S16 once per tile.

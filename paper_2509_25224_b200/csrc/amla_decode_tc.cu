@@ -274,7 +274,12 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
       }
       ext = scale_nn ? fmaxf(ext, ext_b) : fminf(ext, ext_b);
       const float tmax = (nvis > 0) ? ext * prm.scale_log2 : -INFINITY;
-      const RowStep sp = row_step<kMode>(st, tmax, prm.tau);
+      // Lazy reference: a row must move when its maximum exceeds the reference by more than tau.  The correction warp
+      // that serves these 32 rows pays for a rescale as soon as one of them moves, so when one must, every row of the
+      // warp whose maximum rose moves with it (moving early is always allowed: tau = 0 moves at every rise); the rows
+      // then tend to stay in step and the warp rescales on far fewer tiles.
+      const bool must = tmax > st.m2 + prm.tau;
+      const RowStep sp = row_step<kMode>(st, tmax, __any_sync(0xffffffffu, must) ? 0.f : prm.tau);
       // Line 10's factor S16 goes into the exponential's argument (the paper's remark after Algorithm 2):
       // P * S16 = 2^(a - m + log2 S16).  The row sum of line 6 is the sum of the same FP32 values, taken
       // before the bf16 cast and divided by S16 once per tile.
