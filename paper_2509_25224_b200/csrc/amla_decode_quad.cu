@@ -92,6 +92,7 @@ constexpr uint32_t kSmemBytes = kOffSeqlens + kSmemPlanItems * 4;
 #define QSTAMP_NS(smem_base_, idx) do { } while (0)
 #endif
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory a block can opt in to");
+static_assert(kNumP == 4, "the two staging blocks per softmax warp rely on it: the P V awaited before a page is sent is that of the page four back, which used the same block");
 static_assert(kOffK % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 
 constexpr uint32_t kTmemCols = 512;
