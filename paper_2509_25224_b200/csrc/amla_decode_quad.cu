@@ -440,6 +440,10 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
   const uint32_t myV_base = map_to_cta(smem_base, 2 + half);           // score CTA j -> value CTA j
   const uint32_t myV_bars = map_to_cta(bars, 2 + half);
 
+  // The lengths of the first 32 items are requested before anything else, so that their latency runs under the set-up
+  // below (they are inputs of the call: no kernel that this one may overlap with writes them).
+  int early_len = 0;
+  if (wid == 6 && prm.fused_plan && lane < prm.n_items) early_len = prm.seqlens[lane / prm.nrb];
   if (tid == 0) {
     for (int i = 0; i < kNumP; ++i) mbar_init(bar(X_PV + i), 1);
     if (is_score) {
@@ -479,7 +483,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       int carry = 0;
       for (int base = 0; base < prm.n_items; base += 32) {
         const int it = base + lane;
-        const int n_seq = it < prm.n_items ? prm.seqlens[it / prm.nrb] : 0;
+        const int n_seq = it >= prm.n_items ? 0 : base == 0 ? early_len : prm.seqlens[it / prm.nrb];
         if (ps && it < prm.n_items) reinterpret_cast<int*>(smem_raw + kOffSeqlens)[it / prm.nrb] = n_seq;
         const int v = it < prm.n_items ? schedule_length(n_seq, it, prm.tile_keys, prm.ovh) : 0;
         int x = v;
@@ -504,13 +508,12 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     __syncthreads();
     if (ps) { prefix = ps; seqlens = reinterpret_cast<const int*>(smem_raw + kOffSeqlens); }
   }
-  if (is_score && tid < kRowBlock) {
+  if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
     UnitIter first(prm, prefix, seqlens, part);
     Unit fu;
     if (first.next(fu)) prefetch_q_row(prm, fu, half * kRowBlock + tid);
   }
 
-  if (tid == 0) QSTAMP_NS(smem_base, 3);
   bool ok = true;
   UnitIter iter(prm, prefix, seqlens, part);
   Unit u;

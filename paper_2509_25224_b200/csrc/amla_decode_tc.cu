@@ -400,6 +400,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   const uint32_t peerB_base = map_to_cta(smem_base, 1);
   const uint32_t peerA_bars = map_to_cta(smem_base + kOffBars, 0);
 
+  // The lengths of the first 32 items are requested before anything else, so that their latency runs under the set-up
+  // below (they are inputs of the call: no kernel that this one may overlap with writes them).
+  int early_len = 0;
+  if (wid == 6 && prm.fused_plan && lane < prm.n_items) early_len = prm.seqlens[lane / prm.nrb];
   if (tid == 0) {
     for (int i = 0; i < kNumP; ++i) mbar_init(bar(X_PV + i), 1);
     if (is_score) {
@@ -446,7 +450,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       int carry = 0;
       for (int base = 0; base < prm.n_items; base += 32) {
         const int it = base + lane;
-        const int n_seq = it < prm.n_items ? prm.seqlens[it / prm.nrb] : 0;
+        const int n_seq = it >= prm.n_items ? 0 : base == 0 ? early_len : prm.seqlens[it / prm.nrb];
         if (ps && it < prm.n_items) reinterpret_cast<int*>(smem_raw + kOffSeqlens)[it / prm.nrb] = n_seq;   // same value from every row block
         const int v = it < prm.n_items ? schedule_length(n_seq, it, prm.tile_keys, prm.ovh) : 0;
         int x = v;
@@ -471,16 +475,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     __syncthreads();
     if (ps) { prefix = ps; seqlens = reinterpret_cast<const int*>(smem_raw + kOffSeqlens); }
   }
-  if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
-    UnitIter first(prm, prefix, seqlens, part);
-    Unit fu;
-    if (first.next(fu)) prefetch_q_row(prm, fu, tid);
-  }
-
-
+  // Every thread walks its cluster's units; the first one is looked up once, here, and also tells the score CTA(s)
+  // which Q rows to bring into L2 while the roles start.
   bool ok = true;
   UnitIter iter(prm, prefix, seqlens, part);
   Unit u;
+  bool have = wid != 4 && iter.next(u);      // (warp 4, the TMA producers, walk the schedule with cursors of their own and start at once)
+  if (is_score && tid < kRowBlock && have) prefetch_q_row(prm, u, tid);
   uint32_t gt = 0;      // 64-key pages processed by this cluster so far (all roles count identically)
   uint32_t un = 0;      // units processed so far
 
@@ -493,7 +494,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       const int r = tid;
       const uint32_t lane_base = static_cast<uint32_t>(wid * 32) << 16;
       const RoleCtx ctx{smem_base, bars, tbase, peerB_bars, peerB_base, prefix, seqlens, part, tid};
-      while (ok && iter.next(u)) {
+      for (; ok && have; have = iter.next(u)) {
         // Q row -> tensor memory / shared memory (the previous unit's QK^T must be finished with it)
         ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
         if (!ok) break;
@@ -586,7 +587,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         const uint32_t klo0 = smem_desc_lo(smem_base + kOffK, 16);
         const uint32_t qlo0 = smem_desc_lo(smem_base + kOffQRope, 16);
         uint32_t slot = 0, kpar = 0;          // ring position and the parity its "full" barrier completes next
-        while (ok && iter.next(u)) {
+        for (; ok && have; have = iter.next(u)) {
           ok = mbar_wait(bar(A_QREADY), un & 1);
           if (!ok) break;
           tc_fence_after_sync();
@@ -670,7 +671,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         constexpr int kChunks = 17;                         // 512-byte chunks per warp (33 in total)
         const int qr = (wid & 3) * 32 + lane;               // query row whose second half this thread loads
         const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
-        while (ok && iter.next(u)) {
+        for (; ok && have; have = iter.next(u)) {
           {
             ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
             if (!ok) break;
@@ -730,7 +731,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       const int r = (wid & 3) * 32 + lane;
       const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
       const int c_first = partner ? 8 : 0;          // first of this warp's eight 32-column chunks
-      while (ok && iter.next(u)) {
+      for (; ok && have; have = iter.next(u)) {
         int2 info;
         const int slot = partner ? -1 : iter.slot_of(u, &info);
         if (tid == 0) prm.item_info[u.it] = info;
@@ -942,7 +943,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         const uint32_t vlo0 = smem_desc_lo(smem_base + kOffV, kBoxBytes);
         const uint32_t plo0 = smem_desc_lo(smem_base + kOffP, 16);
         uint32_t slot = 0, vpar = 0;
-        while (ok && iter.next(u)) {
+        for (; ok && have; have = iter.next(u)) {
           for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
             const uint32_t s = gt % kNumP, k = gt / kNumP;
             ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
