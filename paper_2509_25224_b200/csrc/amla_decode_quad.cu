@@ -628,7 +628,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
           tc_fence_after_sync();
           for (int t = u.t0; t < u.t1 && ok; ++t, ++gs) {
             const uint32_t sb = gs & 1;
-            ok = mbar_wait<true>(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
+            ok = mbar_wait(bar(A_SEMPTY + sb), ((gs >> 1) & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
             QSTAMP(smem_base, 0, gs);
@@ -646,7 +646,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             }
 #pragma unroll
             for (int gg = 0; gg < 3; ++gg) {
-              ok = ok && (have[gg] || mbar_wait<true>(bar(A_KFULL) + 8 * slot, kpar));
+              ok = ok && (have[gg] || mbar_wait(bar(A_KFULL) + 8 * slot, kpar));
               if (ok) {
                 if (gg == 0) QSTAMP(smem_base, 12, gs);
                 const uint32_t klo = klo0 + slot * (kKSlotBytes >> 4);
@@ -888,12 +888,12 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             ok = mbar_wait<true>(bar(B_PFULL + s), k & 1);
             if (!ok) break;
             QSTAMP(smem_base, 10, gt);
-            ok = mbar_wait<true>(bar(B_OREADY + s), k & 1);
+            ok = mbar_wait(bar(B_OREADY + s), k & 1);
             if (!ok) break;
             QSTAMP(smem_base, 11, gt);
             tc_fence_after_sync();
             fence_proxy_async_smem();
-            ok = mbar_wait<true>(bar(B_VFULL) + 8 * slot, vpar);
+            ok = mbar_wait(bar(B_VFULL) + 8 * slot, vpar);
             if (!ok) break;
             QSTAMP(smem_base, 8, gt);
             const uint32_t plo = plo0 + s * (kPStride >> 4);

@@ -34,7 +34,7 @@ def test_ragged_batch_all_rescale_modes(mode):
     check_full(w, mode)
 
 
-@pytest.mark.parametrize("Sq,H", [(1, 16), (1, 32), (1, 64), (2, 64), (2, 128), (3, 128), (4, 128), (1, 100), (3, 50)])
+@pytest.mark.parametrize("Sq,H", [(1, 16), (1, 32), (1, 64), (2, 64), (2, 128), (3, 128), (4, 128), (1, 100), (3, 50), (5, 100), (8, 128), (8, 17)])
 def test_head_and_token_shapes(Sq, H):
     w = synth.make_workload("s", 3, Sq, H, [200, 77, 513], seed=300 + 10 * Sq + H)
     check_full(w)
@@ -144,6 +144,13 @@ def test_more_items_than_the_in_kernel_schedule_handles():
     # above 2048 (sequence, row block) items the schedule prefix comes from its own kernel instead of the decode kernel
     rng = np.random.default_rng(10)
     w = synth.make_workload("big", 2100, 1, 16, rng.integers(0, 130, 2100), seed=11)
+    check_full(w)
+
+
+def test_more_256_row_items_than_the_in_kernel_schedule_handles():
+    # the same with two query tokens and 128 heads: 2100 items of 256 rows, schedule prefix from its own kernel
+    rng = np.random.default_rng(14)
+    w = synth.make_workload("bigq", 2100, 2, 128, rng.integers(0, 200, 2100), seed=15)
     check_full(w)
 
 
