@@ -174,9 +174,11 @@ __device__ __forceinline__ uint16_t* partial_halves(const DecodeParams& prm) { r
 __device__ __forceinline__ uint8_t* partial_scales(const DecodeParams& prm) {
   return reinterpret_cast<uint8_t*>(prm.part_o) + partial_rows(prm) * kDv * sizeof(uint16_t);
 }
-// scale byte and the factor 2^(127 - byte) for a chunk whose largest magnitude is max_abs
+// scale byte and the factor 2^(127 - byte) for a chunk whose largest magnitude is max_abs.  The byte is the
+// magnitude's exponent field kept within [64, 253]: the factor stays below 2^64, so it can be folded into another
+// finite factor without overflow (chunks below 2^-63 lose precision that nothing downstream can see), and is normal.
 __device__ __forceinline__ uint32_t partial_scale_byte(float max_abs, float* factor) {
-  const uint32_t e = min((__float_as_uint(max_abs) >> 23) & 0xffu, 253u);
+  const uint32_t e = min(max((__float_as_uint(max_abs) >> 23) & 0xffu, 64u), 253u);
   *factor = __uint_as_float((254u - e) << 23);
   return e;
 }

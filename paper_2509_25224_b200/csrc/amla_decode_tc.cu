@@ -27,6 +27,7 @@
 
 #include "amla_common.cuh"
 #include "amla_sm100.cuh"
+#include "amla_epilogue.cuh"
 
 namespace amla {
 
@@ -61,8 +62,7 @@ constexpr uint32_t kVSlotBytes = 4 * kBoxBytes;         // 64 keys x 256 columns
 constexpr uint32_t kOffV = 0;
 constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;    // kNumP x kPStride (P~ then N)
 constexpr uint32_t kOffFin = kOffP + kNumP * kPStride;  // float2 [2][128] (1/(l*S16), lse)
-constexpr uint32_t kOffEpi = kOffFin + 2 * 128 * 8;     // epilogue transpose tiles: 4 warps x 32 rows x 128 B
-constexpr uint32_t kEndB = kOffEpi + 4 * 32 * 128;
+constexpr uint32_t kEndB = kOffFin + 2 * 128 * 8;
 // ---- both: the barriers sit at the same offset, so that one multicast commit can reach the two CTAs
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
 constexpr uint32_t kBarBytes = 512;
@@ -85,7 +85,7 @@ constexpr uint32_t kSCol = 256;          // score CTA: S buffers, 2 x 128 column
 // score CTA the same arrival (multicast commit) frees the page's P buffer for the softmax (PEMPTY).
 enum { X_PV = 0, X_COMMON = X_PV + kNumP };
 enum { A_KFULL = X_COMMON, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2,
-       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2, A_QFREE, A_FINFREE, A_NUM = A_FINFREE + 2 };
+       A_PSTAGED = A_SEMPTY + 2, A_STAGEFREE = A_PSTAGED + 2, A_QREADY = A_STAGEFREE + 2, A_QFREE, A_FINFREE, A_QDONE = A_FINFREE + 2, A_NUM = A_QDONE + kNumKSlots };
 enum { B_VFULL = X_COMMON, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP,
        B_FINFULL = B_OREADY + kNumP, B_NUM = B_FINFULL + 2 };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
@@ -140,12 +140,15 @@ struct Cursor {
   UnitIter it;
   Unit u;
   int base;      // index of the current unit's first page / score tile
+  int ord;       // ordinal of the current unit within the part
   bool valid;
-  __device__ Cursor(const DecodeParams& prm, const int* prefix, const int* seqlens, int part) : it(prm, prefix, seqlens, part), base(0) { valid = it.next(u); }
+  __device__ Cursor(const DecodeParams& prm, const int* prefix, const int* seqlens, int part) : it(prm, prefix, seqlens, part), base(0), ord(0) { valid = it.next(u); }
+  // adopts a walk whose first unit (`first`, if `has_first`) has been looked up already
+  __device__ Cursor(const UnitIter& after_first, const Unit& first, bool has_first) : it(after_first), u(first), base(0), ord(0), valid(has_first) {}
   __device__ int count() const { return kTiles ? (u.t1 - u.t0 + 1) / 2 : (u.t1 - u.t0); }
   // false when k lies beyond the part's work; otherwise `local` is the index within the unit
   __device__ bool locate(int k, int& local) {
-    while (valid && k >= base + count()) { base += count(); valid = it.next(u); }
+    while (valid && k >= base + count()) { base += count(); valid = it.next(u); ++ord; }
     local = k - base;
     return valid;
   }
@@ -169,28 +172,42 @@ __device__ __forceinline__ void prefetch_q_row(const DecodeParams& prm, const Un
   }
 }
 
-// One query row: four 64-column blocks [blk0, blk0 + 4) of its latent part go from global memory into the
-// 128 tensor-memory columns that hold them (two bf16 per column), two blocks at a time.  Every lane reads its own
-// row, so an instruction touches 32 lines; 256-bit loads halve the number of such instructions.
-__device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int blk0, uint32_t taddr) {
-#pragma unroll 1
-  for (int b = blk0; b < blk0 + 4; b += 2) {
-    uint32_t x0[32], x1[32];
-    if (valid) {
+// Q comes on chip through the K ring: at the start of a unit every ring slot takes two 64-column blocks of the unit's
+// 128 rows (TMA boxes, [block][row][128 B] with the 128-byte swizzle), the RoPE block goes straight to its operand tile.
+// Eight warps then move the latent blocks into tensor memory: thread = row, a warp and its partner take one block of
+// the slot each.  This is one block: 128 bytes of the row from the swizzled box into 32 columns (two bf16 per column).
+constexpr uint32_t kQBlockBytes = 128 * 128;            // one 64-column block of 128 rows
+__device__ __forceinline__ void move_q_block(uint32_t box, int row, bool valid, uint32_t taddr) {
+  uint32_t x[32];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        ldg_256(qrow + b * 8 + 2 * c, x0, 8 * c);
-        ldg_256(qrow + b * 8 + 8 + 2 * c, x1, 8 * c);
-      }
-    } else {
+  for (int c = 0; c < 8; ++c)
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x[4 * c]), "=r"(x[4 * c + 1]), "=r"(x[4 * c + 2]), "=r"(x[4 * c + 3])
+                 : "r"(box + sw128_offset(row, c)));
+  if (!valid) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) { x0[i] = 0; x1[i] = 0; }
-    }
-    tmem_st_32x32b_x32(taddr + b * 32, x0);
-    tmem_st_32x32b_x32(taddr + b * 32 + 32, x1);
+    for (int i = 0; i < 32; ++i) x[i] = 0;
   }
+  tmem_st_32x32b_x32(taddr, x);
 }
 
+// The eight Q warps' share of a unit's start: wait for each slot's piece, move it, hand the slot back.  `gs` = score
+// tiles of this cluster before the unit (three K slots each), `un` = units before it: slot e has completed
+// un + ceil((3 gs - e) / 4) phases so far.  Returns false after a timeout.
+__device__ __forceinline__ bool move_q_unit(const DecodeParams& prm, int part, uint32_t smem_base, uint32_t bars, uint32_t taddr_row, int row, bool valid, int blk,
+                                            uint32_t un, uint32_t gs, int lane) {
+  bool ok = true;
+#pragma unroll 1
+  for (int e = 0; e < kNumKSlots && ok; ++e) {
+    const uint32_t par = (un + (3 * gs + 3 - e) / 4) & 1;
+    ok = __all_sync(0xffffffffu, mbar_wait(bars + 8u * (A_KFULL + e), par));
+    if (!ok) break;
+    if (row == 0) AMLA_STAMP2(prm, part, 28 + blk, un * kNumKSlots + e);
+    move_q_block(smem_base + kOffK + e * kKSlotBytes + blk * kQBlockBytes, row, valid, taddr_row + 32 * (2 * e + blk));
+    __syncwarp();                                       // every lane's reads of the slot are done
+    if (lane == 0) mbar_arrive(bars + 8u * (A_QDONE + e));
+  }
+  return ok;
+}
 
 // What a role needs from the kernel's set-up.
 struct RoleCtx {
@@ -380,7 +397,8 @@ __device__ __noinline__ uint64_t softmax_unit(const DecodeParams prm, const Role
 
 template <int kMode, bool kGuard>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap v_map, const DecodeParams prm) {
+decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap q_map,
+                 const DecodeParams prm) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t smem_base = smem_u32(smem_raw);
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
@@ -414,7 +432,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       }
       mbar_init(bar(A_QREADY), 256);
       mbar_init(bar(A_QFREE), 1);
-      for (int i = 0; i < 2; ++i) mbar_init(bar(A_FINFREE + i), 4);   // the four epilogue warps of the value CTA
+      for (int i = 0; i < kNumKSlots; ++i) mbar_init(bar(A_QDONE + i), 8);   // the eight warps that move Q on chip
+      for (int i = 0; i < 2; ++i) mbar_init(bar(A_FINFREE + i), 8);   // the eight epilogue warps of the value CTA
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
       for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), 256); }
@@ -423,6 +442,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     fence_mbar_init();
     prefetch_tensormap(&kv_map);
     prefetch_tensormap(&v_map);
+    prefetch_tensormap(&q_map);
   }
   if (wid == 5) { tmem_alloc(tmem_slot, kTmemCols); tmem_relinquish(); }
   tc_fence_before_sync();
@@ -480,8 +500,19 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   bool ok = true;
   UnitIter iter(prm, prefix, seqlens, part);
   Unit u;
-  bool have = wid != 4 && iter.next(u);      // (warp 4, the TMA producers, walk the schedule with cursors of their own and start at once)
-  if (is_score && tid < kRowBlock && have) prefetch_q_row(prm, u, tid);
+  bool have = iter.next(u);
+  // The first unit's Q is requested here, by the first thread that knows the unit: the producer lanes reach their
+  // first load thousands of cycles later (their start-up code is longer and runs from a cold instruction cache).
+  if (is_score && tid == 0 && have) {
+    const int row = u.b * prm.R + u.r0;
+    for (int l = 0; l < kNumKSlots; ++l) {
+      const uint32_t full = bar(A_KFULL + l), dst = smem_base + kOffK + l * kKSlotBytes;
+      mbar_arrive_expect_tx(full, (l == 0 ? 3 : 2) * kQBlockBytes);
+      tma_load_3d(dst, &q_map, 0, row, 2 * l, full);
+      tma_load_3d(dst + kQBlockBytes, &q_map, 0, row, 2 * l + 1, full);
+      if (l == 0) tma_load_3d(smem_base + kOffQRope, &q_map, 0, row, 8, full);
+    }
+  }
   uint32_t gt = 0;      // 64-key pages processed by this cluster so far (all roles count identically)
   uint32_t un = 0;      // units processed so far
 
@@ -500,14 +531,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         if (!ok) break;
         tc_fence_after_sync();
         if (tid == 0) AMLA_STAMP(prm, part, 10, un);
-        {
-          // this warpgroup brings in the first 256 latent columns of its rows; the copy warps, idle at this
-          // point, bring in the other 256 and the RoPE columns
-          const bool valid = r < u.nrows;
-          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDqk);
-          load_q_latent(qrow, valid, 0, tbase + lane_base + kQCol);
-          tmem_wait_st();
-        }
+        // this warpgroup moves the first block of every slot's piece of Q, the copy warps (idle at this point) the second
+        ok = move_q_unit(prm, part, smem_base, bars, tbase + lane_base + kQCol, r, r < u.nrows, 0, un, gs, lane);
+        if (!ok) break;
+        tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(bar(A_QREADY));
         if (tid == 0) AMLA_STAMP(prm, part, 11, un);
@@ -520,47 +547,88 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       }
       if (!ok) report_timeout(prm.status);
     } else if (wid == 4) {
-      // ---- TMA producers: K, three slots (192 columns each) per score tile.  Lane l owns ring slot l and
-      // loads every kNumKSlots-th slot of the sequence; the lanes poll without blocking, so that a slot that
-      // is still in use never holds up the loads of the others (one thread issuing a ring in order reaches a
-      // fraction of the rate).
+      // ---- TMA producers.  Lane l owns ring slot l.  The slot carries, in this order: the lane's piece of Q at the
+      // start of every unit (two 64-column blocks; lane 0 adds the RoPE block, which goes straight to its operand tile
+      // once the previous unit's MMAs have let go of it), and every kNumKSlots-th K slot of the sequence (three slots
+      // of 192 columns per score tile).  The lanes poll without blocking, so that a slot that is still in use never
+      // holds up the loads of the others (one thread issuing a ring in order reaches a fraction of the rate).
       {
-        Cursor<true> cur(prm, prefix, seqlens, part);
-        int my_tile = lane / 3, g = lane % 3;   // score tile and column-block group of the next slot this lane loads
-        uint32_t par = 1;                       // parity of the "empty" phase it has to see first
-        bool fin = lane >= kNumKSlots, have = false;
+        // The first unit has been looked up and its Q requested before the roles split; the way to this lane's first
+        // K load is kept short (no further look-up before it; the next unit's is made when it is first asked for).
+        bool fin = lane >= kNumKSlots;
+        const bool first_out = !fin && have;
+        Cursor<true> cur(iter, u, have);
+        UnitIter qit = iter;                    // walks the units whose Q this lane has not loaded:
+        Unit qu;                                //   qu = the next one (valid once looked up), q_ord its ordinal
+        bool q_left = false, q_stale = first_out;
+        auto q_due = [&]() { if (q_stale) { q_left = qit.next(qu); q_stale = false; } return q_left; };
+        int q_ord = first_out ? 1 : 0;
+        int my_tile = lane / 3, g = lane % 3;   // score tile and column-block group of the next K slot this lane loads
+        int k_state = 0;                        // 0: not looked up, 1: page numbers at hand, 2: no K slot left
+        int k_ord = 0;
+        int pending = 0;                        // 0: decide, 1: a piece of Q, 2: a K slot
+        int last = first_out ? 1 : 0;           // what the slot holds now (same code): tells which barrier frees it
         int page0 = 0, page1 = 0, npages = 0;
-        int issued = 0;
-        const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane);
+        int nq = first_out ? 1 : 0, nk = 0;     // pieces of Q / K slots issued for this lane's slot
+        const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane), my_qdone = bar(A_QDONE + lane);
         const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
         uint64_t t_start = global_timer_ns();     // restarted whenever a lane issues a load: the limit bounds one stalled wait
         bool progress = false;
         for (uint32_t spin = 0;; ++spin) {
-          if (!fin && !have) {
-            int lt;
-            if (cur.locate(my_tile, lt)) {
-              const int t = cur.u.t0 + 2 * lt;
-              const int32_t* bt = prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq;
-              npages = min(2, cur.u.t1 - t);
-              page0 = __ldg(bt + t);
-              page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
-              have = true;
-            } else {
-              fin = true;
+          if (!fin && pending == 0) {
+            // (the cursor's unit is never behind the unit of the next K slot: when Q is due by that count, it goes out
+            // before the K slot is looked up -- the unit's first load should not wait for a block-table entry)
+            if (q_ord <= cur.ord && q_due()) pending = 1;
+            else if (k_state == 0) {
+              int lt;
+              if (cur.locate(my_tile, lt)) {
+                const int t = cur.u.t0 + 2 * lt;
+                const int32_t* bt = prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq;
+                npages = min(2, cur.u.t1 - t);
+                page0 = __ldg(bt + t);
+                page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
+                k_ord = cur.ord;
+                k_state = 1;
+              } else {
+                k_state = 2;
+              }
+            }
+            if (pending == 0) {
+              if ((k_state == 2 || q_ord <= k_ord) && q_due()) pending = 1;
+              else if (k_state == 1) pending = 2;
+              else if (k_state == 2) fin = true;
             }
           }
-          if (have && mbar_probe(my_empty, par)) {
-            AMLA_STAMP2(prm, part, 20, issued * kNumKSlots + lane);
-            mbar_arrive_expect_tx(my_full, npages * kKPageBytes);
-            tma_load_4d(dst, &kv_map, 0, 0, 3 * g, page0 * 8, my_full);
-            if (npages > 1) tma_load_4d(dst + kKPageBytes, &kv_map, 0, 0, 3 * g, page1 * 8, my_full);
-            // kNumKSlots slots further on
-            g += kNumKSlots % 3; my_tile += kNumKSlots / 3;
-            if (g >= 3) { g -= 3; my_tile += 1; }
-            par ^= 1;
-            ++issued;
-            have = false;
-            progress = true;
+          if (pending != 0) {
+            // the slot's previous content has been used up: a piece of Q by the eight Q warps, a K slot by its MMAs
+            bool free_now = last == 0 || (last == 1 ? mbar_probe(my_qdone, (nq - 1) & 1) : mbar_probe(my_empty, (nk - 1) & 1));
+            if (free_now && pending == 1 && lane == 0 && q_ord > 0) free_now = mbar_probe(bar(A_QFREE), (q_ord - 1) & 1);
+            if (free_now) {
+              if (pending == 1) {
+                const int row = qu.b * prm.R + qu.r0;
+                AMLA_STAMP2(prm, part, 27, q_ord * kNumKSlots + lane);
+                mbar_arrive_expect_tx(my_full, (lane == 0 ? 3 : 2) * kQBlockBytes);
+                tma_load_3d(dst, &q_map, 0, row, 2 * lane, my_full);
+                tma_load_3d(dst + kQBlockBytes, &q_map, 0, row, 2 * lane + 1, my_full);
+                if (lane == 0) tma_load_3d(smem_base + kOffQRope, &q_map, 0, row, 8, my_full);
+                q_stale = true;
+                ++q_ord; ++nq;
+                last = 1;
+              } else {
+                AMLA_STAMP2(prm, part, 20, nk * kNumKSlots + lane);
+                mbar_arrive_expect_tx(my_full, npages * kKPageBytes);
+                tma_load_4d(dst, &kv_map, 0, 0, 3 * g, page0 * 8, my_full);
+                if (npages > 1) tma_load_4d(dst + kKPageBytes, &kv_map, 0, 0, 3 * g, page1 * 8, my_full);
+                // kNumKSlots slots further on
+                g += kNumKSlots % 3; my_tile += kNumKSlots / 3;
+                if (g >= 3) { g -= 3; my_tile += 1; }
+                ++nk;
+                k_state = 0;
+                last = 2;
+              }
+              pending = 0;
+              progress = true;
+            }
           }
           if (__all_sync(0xffffffffu, fin)) break;
           // nothing to issue right now: back off, so that the polling does not take issue slots from the warps that
@@ -572,7 +640,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         if (!ok) {
           if (lane == 0) report_timeout(prm.status);
           // let the copy that may still be in flight land before the CTA exits
-          if (issued > 0 && lane < kNumKSlots) mbar_wait(my_full, (issued - 1) & 1);
+          if (nq + nk > 0 && lane < kNumKSlots) mbar_wait(my_full, (nq + nk - 1) & 1);
         }
       }
     } else if (wid == 5) {
@@ -591,6 +659,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           ok = mbar_wait(bar(A_QREADY), un & 1);
           if (!ok) break;
           tc_fence_after_sync();
+          kpar ^= 1;                          // the unit's pieces of Q have been through every slot once
           for (int t = u.t0; t < u.t1 && ok; t += 2, ++gs) {
             const int npages = min(2, u.t1 - t);
             const uint32_t idesc = npages > 1 ? idesc128 : idesc64;
@@ -639,19 +708,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
       }
 #ifdef AMLA_TRACE
     } else if (wid == 6 + kNumCopyWarps) {
-      // trace builds: lane l watches K slot l and stamps the arrival of its data (non-blocking polls)
+      // trace builds: lanes 4-7 stamp the phases of the S barriers (non-blocking polls)
       if (prm.trace) {
         Cursor<true> cur(prm, prefix, seqlens, part);
         int total = 0, lt;
         while (cur.valid) { total += cur.count(); cur.locate(total, lt); }
         total *= 3;
         uint32_t par = 0;
-        int g = lane;
         int gs2 = lane & 1;                       // lanes 4..7: score tile whose SFULL (4, 5) / SEMPTY (6, 7) phase comes next
         const uint64_t t_start = global_timer_ns();
         for (uint32_t spin = 0;; ++spin) {
-          const bool act = lane < kNumKSlots && g < total;
-          if (act && mbar_probe(bar(A_KFULL + lane), par)) { AMLA_STAMP2(prm, part, 24, g); g += kNumKSlots; par ^= 1; }
+          const bool act = false;
           const bool act2 = lane >= 4 && lane < 8 && gs2 < total / 3;
           if (act2 && mbar_probe(bar((lane < 6 ? A_SFULL : A_SEMPTY) + (lane & 1)), par)) { AMLA_STAMP2(prm, part, lane < 6 ? 30 : 31, gs2); gs2 += 2; par ^= 1; }
           if (!__any_sync(0xffffffffu, act || act2)) break;
@@ -671,21 +738,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
         constexpr int kChunks = 17;                         // 512-byte chunks per warp (33 in total)
         const int qr = (wid & 3) * 32 + lane;               // query row whose second half this thread loads
         const uint32_t q_lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
+        uint32_t gs_c = 0;                                  // score tiles before the current unit
         for (; ok && have; have = iter.next(u)) {
           {
             ok = warp_wait(bar(A_QFREE), (un & 1) ^ 1);
             if (!ok) break;
             tc_fence_after_sync();
-            const bool valid = qr < u.nrows;
-            const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? qr : 0)) * kDqk);
-            load_q_latent(qrow, valid, 4, tbase + q_lane_base + kQCol);
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-              const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
-              st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
-            }
+            ok = move_q_unit(prm, part, smem_base, bars, tbase + q_lane_base + kQCol, qr, qr < u.nrows, 1, un, gs_c, lane);
+            if (!ok) break;
+            gs_c += (u.t1 - u.t0 + 1) >> 1;
             tmem_wait_st();
-            fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(bar(A_QREADY));
             ++un;
@@ -726,14 +788,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     if (wid < 4 || (wid >= 6 && wid < 10)) {
       // ---- correction + epilogue warpgroup: thread = query row.  A warp reaches the tensor-memory lanes
       // 32 * (warp % 4) .. + 31, so warps 6-9, which have no other work in this CTA, are the partners of warps 2, 3,
-      // 0, 1: each of a pair rescales one half of the row's 512 columns.  The epilogue stays with warps 0-3.
+      // 0, 1: each of a pair takes one half of the row's 512 columns, in the rescale and in the epilogue.
       const bool partner = wid >= 4;
       const int r = (wid & 3) * 32 + lane;
       const uint32_t lane_base = static_cast<uint32_t>((wid & 3) * 32) << 16;
       const int c_first = partner ? 8 : 0;          // first of this warp's eight 32-column chunks
       for (; ok && have; have = iter.next(u)) {
         int2 info;
-        const int slot = partner ? -1 : iter.slot_of(u, &info);
+        const int slot = iter.slot_of(u, &info);
         if (tid == 0) prm.item_info[u.it] = info;
         for (int t = u.t0; t < u.t1 && ok; ++t, ++gt) {
           const uint32_t s = gt % kNumP, k = gt / kNumP;
@@ -796,8 +858,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           if (tid == 0) AMLA_STAMP2(prm, part, 14, gt);
         }
         if (!ok) break;
-        // ---- epilogue (line 20): out = O / (l * S16)
-        if (!partner) {
+        // ---- epilogue (line 20): out = O / (l * S16).  Thread = row; a warp and its partner take eight 32-column
+        // chunks each, scale them and store them from registers with 256-bit stores (a full 32-byte sector per lane).  An SM
+        // writes about 32 B per clock whatever the instruction: the 128 KB of a unit take 4-5 thousand clocks, and staging
+        // them for tiled TMA stores (64-byte or 32-byte rows) was no faster.
+        {
           const uint32_t gl = gt - 1;
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
@@ -814,75 +879,40 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster_relaxed(peerA_bars + 8u * (A_FINFREE + (un & 1)));   // the entry may be rewritten
           const bool valid = r < u.nrows;
-          // 32 columns at a time: each lane scales its row, the warp transposes the 32 x 32 tile through shared
-          // memory (16-byte units XOR-swizzled by row), and writes whole 128-byte (FP32 partial) or 64-byte (bf16)
-          // row pieces, so that a store instruction covers full lines instead of 32 scattered sectors.
-          const uint32_t epi = smem_base + kOffEpi + wid * (32 * 128);
-          const int rows_here = min(32, u.nrows - wid * 32);          // valid rows of this warp's 32 (may be <= 0)
-          __nv_bfloat16* obase = prm.out + (static_cast<size_t>(u.b) * prm.R + u.r0 + wid * 32) * kDv;
-          const size_t prow0 = static_cast<size_t>(slot < 0 ? 0 : slot) * kRowBlock + wid * 32;   // this warp's first row of the partial arrays
-          uint16_t* hbase = partial_halves(prm) + prow0 * kDv;
-          unsigned long long sc_lo = 0, sc_hi = 0;                    // this thread's row: sixteen scale bytes
+          const size_t prow = static_cast<size_t>(slot < 0 ? 0 : slot) * kRowBlock + r;   // row of the partial arrays
+          uint32_t sc_lo = 0, sc_hi = 0;                                  // this thread's eight scale bytes
+          uint16_t* orow = reinterpret_cast<uint16_t*>(prm.out) + (static_cast<size_t>(u.b) * prm.R + u.r0 + (valid ? r : 0)) * kDv;
+          uint16_t* hrow = partial_halves(prm) + prow * kDv;
           uint32_t o[2][32];
-          tmem_ld_32x32b_x32(tbase + lane_base, o[0]);
+          tmem_ld_32x32b_x32(tbase + lane_base + 32 * c_first, o[0]);
 #pragma unroll 1
-          for (int c = 0; c < 16; c += 2) {
+          for (int cq = 0; cq < 8; cq += 2) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               tmem_wait_ld();
-              if (c + e + 1 < 16) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (c + e + 1), o[e ^ 1]);
-              const int cc = c + e;
-              __syncwarp();                                           // the tile is free again (previous read-back done)
+              if (cq + e + 1 < 8) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (c_first + cq + e + 1), o[e ^ 1]);
+              const int cc = c_first + cq + e;
+              uint32_t w[16];
+              uint16_t* dst;
               if (slot < 0) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const uint32_t w0 = pack_bf16x2(__uint_as_float(o[e][8 * j + 0]) * inv, __uint_as_float(o[e][8 * j + 1]) * inv);
-                  const uint32_t w1 = pack_bf16x2(__uint_as_float(o[e][8 * j + 2]) * inv, __uint_as_float(o[e][8 * j + 3]) * inv);
-                  const uint32_t w2 = pack_bf16x2(__uint_as_float(o[e][8 * j + 4]) * inv, __uint_as_float(o[e][8 * j + 5]) * inv);
-                  const uint32_t w3 = pack_bf16x2(__uint_as_float(o[e][8 * j + 6]) * inv, __uint_as_float(o[e][8 * j + 7]) * inv);
-                  st_shared_v4(epi + lane * 128 + ((j ^ (lane & 7)) << 4), w0, w1, w2, w3);
-                }
-                __syncwarp();
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {                         // 8 rows x 64 B per instruction
-                  const int row = 8 * k + (lane >> 2), j = lane & 3;
-                  uint4 v;
-                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                               : "r"(epi + row * 128 + ((j ^ (row & 7)) << 4)));
-                  if (row < rows_here) *reinterpret_cast<uint4*>(obase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * j) = v;
-                }
+                epilogue_chunk_bf16(o[e], inv, w);
+                dst = orow + 32 * cc;
               } else {
-                // split unit: half precision with the chunk's power-of-two scale (see "Split partials")
-                float x[32], mx = 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) { x[j] = __uint_as_float(o[e][j]) * inv; mx = fmaxf(mx, fabsf(x[j])); }
-                float f;
-                const uint32_t sb = partial_scale_byte(mx, &f);
-                if (cc < 8) sc_lo |= static_cast<unsigned long long>(sb) << (8 * cc); else sc_hi |= static_cast<unsigned long long>(sb) << (8 * (cc - 8));
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                  st_shared_v4(epi + lane * 128 + ((j ^ (lane & 7)) << 4),
-                               pack_f16x2(x[8 * j + 0] * f, x[8 * j + 1] * f), pack_f16x2(x[8 * j + 2] * f, x[8 * j + 3] * f),
-                               pack_f16x2(x[8 * j + 4] * f, x[8 * j + 5] * f), pack_f16x2(x[8 * j + 6] * f, x[8 * j + 7] * f));
-                __syncwarp();
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {                         // 8 rows x 64 B per instruction
-                  const int row = 8 * k + (lane >> 2), j = lane & 3;
-                  uint4 v;
-                  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                               : "r"(epi + row * 128 + ((j ^ (row & 7)) << 4)));
-                  if (row < rows_here) *reinterpret_cast<uint4*>(hbase + static_cast<size_t>(row) * kDv + 32 * cc + 8 * j) = v;
-                }
+                const uint32_t sb = epilogue_chunk_partial(o[e], inv, w);
+                if (cq + e < 4) sc_lo |= sb << (8 * (cq + e)); else sc_hi |= sb << (8 * (cq + e - 4));
+                dst = hrow + 32 * cc;
+              }
+              if (valid) {
+                stg_256(dst, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                stg_256(dst + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
               }
             }
           }
-          if (valid) {
-            if (slot < 0) {
-              prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
-            } else {
-              prm.part_lse[static_cast<size_t>(slot) * kRowBlock + r] = lse;
-              *reinterpret_cast<uint4*>(partial_scales(prm) + (static_cast<size_t>(slot) * kRowBlock + r) * 16) = make_uint4(static_cast<uint32_t>(sc_lo), static_cast<uint32_t>(sc_lo >> 32), static_cast<uint32_t>(sc_hi), static_cast<uint32_t>(sc_hi >> 32));
-            }
+          if (valid && slot >= 0)
+            *reinterpret_cast<uint2*>(partial_scales(prm) + prow * 16 + c_first) = make_uint2(sc_lo, sc_hi);
+          if (valid && !partner) {
+            if (slot < 0) prm.lse[static_cast<size_t>(u.b) * prm.R + u.r0 + r] = lse;
+            else prm.part_lse[prow] = lse;
           }
           tc_fence_before_sync();
           if (tid == 0) AMLA_STAMP(prm, part, 19, un);
@@ -893,7 +923,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     } else if (wid == 4) {
       // ---- TMA producers: V, two ring slots per page (256 columns each, one 3-D box per slot); lane l owns ring slot l
       {
-        Cursor<false> cur(prm, prefix, seqlens, part);
+        Cursor<false> cur(iter, u, have);
         int my_gv = lane;                       // next slot of the sequence this lane loads (page = gv / 2)
         uint32_t par = 1;
         bool fin = lane >= kNumVSlots, have = false;
@@ -1009,7 +1039,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 template <int kMode, bool kGuard>
-cudaError_t launch_variant(const CUtensorMap& map, const CUtensorMap& vmap, const DecodeParams& prm, cudaStream_t stream) {
+cudaError_t launch_variant(const CUtensorMap& map, const CUtensorMap& vmap, const CUtensorMap& qmap, const DecodeParams& prm, cudaStream_t stream) {
   auto kern = decode_tc_kernel<kMode, kGuard>;
   // the opt-in to large dynamic shared memory is per device and per kernel; do it once each
   static std::atomic<uint64_t> done{0};
@@ -1032,7 +1062,7 @@ cudaError_t launch_variant(const CUtensorMap& map, const CUtensorMap& vmap, cons
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, map, vmap, prm);
+  return cudaLaunchKernelEx(&cfg, kern, map, vmap, qmap, prm);
 }
 
 }  // namespace
@@ -1069,11 +1099,25 @@ cudaError_t launch_decode_tc(const DecodeParams& prm, cudaStream_t stream, int* 
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (vr != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
+  // Q: (64 columns, rows of all sequences, 9 column blocks); one box = a unit's 128 rows x one column block, laid out
+  // [row][64 columns] like an operand tile.  Rows past the end of the array read as zero; rows of a following
+  // sequence that a short unit's box covers are dropped by the kernel.
+  CUtensorMap qmap;
+  {
+    const cuuint64_t qdims[3] = {64, static_cast<cuuint64_t>(prm.B) * prm.R, static_cast<cuuint64_t>(kDqk / 64)};
+    const cuuint64_t qstrides[2] = {static_cast<cuuint64_t>(kDqk) * 2, 128};
+    const cuuint32_t qbox[3] = {64, kRowBlock, 1};
+    const cuuint32_t qestr[3] = {1, 1, 1};
+    const CUresult qr = encode(&qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(prm.q), qdims, qstrides,
+                               qbox, qestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (qr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
   const int mode = prm.flags & 3;
   const bool guard = !(prm.flags & 4);
-  if (mode == 0) return guard ? launch_variant<0, true>(map, vmap, prm, stream) : launch_variant<0, false>(map, vmap, prm, stream);
-  if (mode == 1) return guard ? launch_variant<1, true>(map, vmap, prm, stream) : launch_variant<1, false>(map, vmap, prm, stream);
-  return launch_variant<2, true>(map, vmap, prm, stream);
+  if (mode == 0) return guard ? launch_variant<0, true>(map, vmap, qmap, prm, stream) : launch_variant<0, false>(map, vmap, qmap, prm, stream);
+  if (mode == 1) return guard ? launch_variant<1, true>(map, vmap, qmap, prm, stream) : launch_variant<1, false>(map, vmap, qmap, prm, stream);
+  return launch_variant<2, true>(map, vmap, qmap, prm, stream);
 }
 
 }  // namespace amla
