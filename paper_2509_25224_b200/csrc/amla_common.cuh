@@ -80,7 +80,10 @@ constexpr int kTraceTiles = 96;
 // L = prefix[n_items] the total, and part p owns positions [p*L/P, (p+1)*L/P).  A part does the
 // tiles whose positions it owns; overhead positions carry no work.
 // ---------------------------------------------------------------------------------------------
-constexpr int kUnitOverheadTiles = 10;        // 128-row kernel: in 64-key pages
+#ifndef AMLA_UNIT_OVERHEAD_TILES
+#define AMLA_UNIT_OVERHEAD_TILES 6            // 128-row kernel: in 64-key pages (a build-time knob for tuning runs)
+#endif
+constexpr int kUnitOverheadTiles = AMLA_UNIT_OVERHEAD_TILES;
 #ifndef AMLA_QUAD_OVERHEAD_TILES
 #define AMLA_QUAD_OVERHEAD_TILES 5            // 256-row kernel: in 128-key tiles (a build-time knob for tuning runs)
 #endif

@@ -33,6 +33,16 @@ namespace amla {
 
 using namespace sm100;
 
+// trace builds: wall-clock stamps (global timer, ns) of a CTA's phases, in event row 31, columns 88..95
+#ifdef AMLA_TRACE
+#define AMLA_STAMP_NS(prm, part, col)                                                                               \
+  do {                                                                                                              \
+    if ((prm).trace) (prm).trace[(static_cast<size_t>(part) * kTraceEvents + 31) * kTraceTiles + (col)] = global_timer_ns(); \
+  } while (0)
+#else
+#define AMLA_STAMP_NS(prm, part, col) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int kNumCopyWarps = 4;         // score CTA: warps that move staged P~ to the value CTA
@@ -410,6 +420,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
     return;
   }
 
+  if (tid == 0) AMLA_STAMP_NS(prm, part, is_score ? 88 : 92);        // entry
   const uint32_t bars = smem_base + kOffBars;
   auto bar = [&](int i) { return bars + 8u * i; };
   const uint32_t tmem_slot = bars + kBarBytes - 8;
@@ -458,6 +469,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   // workspace) are complete after this wait.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;");
+  if (tid == 0) AMLA_STAMP_NS(prm, part, is_score ? 89 : 93);        // the kernel before has completed
   const int* prefix = prm.prefix;
   const int* seqlens = prm.seqlens;
   if (prm.fused_plan) {
@@ -501,6 +513,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   UnitIter iter(prm, prefix, seqlens, part);
   Unit u;
   bool have = iter.next(u);
+  // The producers' first block-table entries: brought into L1 now, ahead of the burst of Q, K and V requests that
+  // starts below (a load that misses during that burst comes back thousands of cycles later, and a producer lane that
+  // waits for one holds up the other lanes of its warp).
+  if (wid == 4 && lane == 0 && have) {
+    const int32_t* bt = prm.block_table + static_cast<size_t>(u.b) * prm.max_blocks_per_seq;
+    prefetch_l1(bt + u.t0);
+    prefetch_l1(bt + min(u.t0 + 32, u.t1 - 1));
+  }
   // The first unit's Q is requested here, by the first thread that knows the unit: the producer lanes reach their
   // first load thousands of cycles later (their start-up code is longer and runs from a cold instruction cache).
   if (is_score && tid == 0 && have) {
@@ -587,7 +607,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
                 npages = min(2, cur.u.t1 - t);
                 page0 = __ldg(bt + t);
                 page1 = npages > 1 ? __ldg(bt + t + 1) : 0;
+                prefetch_l1(bt + min(t + 32, cur.u.t1 - 1));     // the line after this one, well before it is needed
                 k_ord = cur.ord;
+                if (nk == 0) AMLA_STAMP2(prm, part, 27, 64 + lane);
                 k_state = 1;
               } else {
                 k_state = 2;
@@ -937,7 +959,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
           if (!fin && !have) {
             int lt;
             if (cur.locate(my_gv >> 1, lt)) {
-              page = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + cur.u.t0 + lt);
+              const int32_t* bt = prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq;
+              page = __ldg(bt + cur.u.t0 + lt);
+              prefetch_l1(bt + min(cur.u.t0 + lt + 32, cur.u.t1 - 1));
               have = true;
             } else {
               fin = true;
@@ -1012,9 +1036,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap kv_map, const __grid_consta
   // teardown: nobody may still be writing into a peer that has exited
   tc_fence_before_sync();
   __syncthreads();
+  if (tid == 0) AMLA_STAMP_NS(prm, part, is_score ? 90 : 94);        // roles done
   cluster_arrive();
   cluster_wait();
   if (wid == 5) tmem_dealloc(tbase, kTmemCols);
+  if (tid == 0) AMLA_STAMP_NS(prm, part, is_score ? 91 : 95);        // exit
 }
 
 // ---------------------------------------------------------------------------------------------------

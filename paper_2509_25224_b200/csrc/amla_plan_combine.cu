@@ -60,6 +60,9 @@ __global__ void __launch_bounds__(128) combine_kernel(DecodeParams prm) {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_ns));
   if (prm.trace && blockIdx.x == 0 && threadIdx.x == 0) prm.trace[148 * 16 * 128 + 0] = t_ns & 0xffffffffull;
 #endif
+  // A decode kernel that follows on the stream may set itself up beside this kernel (it writes nothing this kernel
+  // reads before its own wait for this kernel's completion).
+  asm volatile("griddepcontrol.launch_dependents;");
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row_global = blockIdx.x * warps_per_block + (threadIdx.x >> 5);

@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _variant(Sq, H):
     """(rows per item, keys per tile, overhead positions) of the schedule for a shape: up to 128 query rows per
     sequence the items are 128-row blocks with one-page tiles, above that 256-row blocks with two-page tiles."""
-    return (256, 128, 5) if Sq * H > 128 else (128, 64, 10)
+    return (256, 128, 5) if Sq * H > 128 else (128, 64, 6)
 
 
 @pytest.fixture(scope="module")
@@ -120,8 +120,8 @@ def test_plan_covers_every_tile_once_and_balances(lib, P):
 
 
 def test_plan_small_case_by_hand(lib):
-    # two sequences of 3 and 1 tiles, 2 parts: positions [tiles 0-2 | 10 overhead, tile 0] = 14; part 0 = [0,7) holds
-    # the first item, part 1 = [7,14) the second
+    # two sequences of 3 and 1 tiles, 2 parts: positions [tiles 0-2 | 6 overhead, tile 0] = 10; part 0 = [0,5) holds
+    # the first item, part 1 = [5,10) the second
     u = binding.plan_host(np.array([129, 10]), 1, 128, 2)
     assert u.tolist() == [[0, 0, 0, 3, -1, 1], [1, 1, 0, 1, -1, 1]]
 
