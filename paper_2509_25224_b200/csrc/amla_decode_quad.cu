@@ -61,7 +61,7 @@ constexpr uint32_t kOffP = kNumVSlots * kVSlotBytes;
 constexpr uint32_t kEndB = kOffP + kNumP * kPStride;
 // ---- all four: barriers at the same offset, so that one multicast commit reaches them
 constexpr uint32_t kOffBars = kEndA > kEndB ? kEndA : kEndB;
-constexpr uint32_t kBarBytes = 256;
+constexpr uint32_t kBarBytes = 320;
 #ifdef AMLA_TRACE
 constexpr int kSmemPlanItems = 4;                    // trace builds: the room goes to the stamps
 #else
@@ -107,7 +107,7 @@ constexpr uint16_t kMaskScore = 0x3, kMaskValue = 0xC, kMaskAll = 0xF;
 // and in the odd CTA the otherwise idle warp 5 relays each completed phase as ONE arrival on the even CTA's copy.
 enum { X_PV = 0, X_COMMON = X_PV + kNumP };
 enum { A_KFULL = X_COMMON /* even CTA */, A_KEMPTY = A_KFULL + kNumKSlots, A_SFULL = A_KEMPTY + kNumKSlots, A_SEMPTY = A_SFULL + 2 /*R*/,
-       A_XCHG = A_SEMPTY + 2, A_QREADY = A_XCHG + 4 /*R*/, A_QFREE, A_NUM };
+       A_XCHG = A_SEMPTY + 2, A_QREADY = A_XCHG + 4 /*R*/, A_QFREE, A_QFULL, A_QDONE = A_QFULL + kNumKSlots, A_NUM = A_QDONE + kNumKSlots };
 enum { B_VFULL = X_COMMON /* even CTA */, B_VEMPTY = B_VFULL + kNumVSlots, B_PFULL = B_VEMPTY + kNumVSlots, B_OREADY = B_PFULL + kNumP /*R*/,
        B_NUM = B_OREADY + kNumP };
 static_assert(A_NUM * 8 + 8 <= kBarBytes && B_NUM * 8 + 8 <= kBarBytes, "barrier area too small");
@@ -158,10 +158,11 @@ struct Cursor {
   UnitIter it;
   Unit u;
   int base;
+  int ord;       // ordinal of the current unit within the part
   bool valid;
-  __device__ Cursor(const DecodeParams& prm, const int* prefix, const int* seqlens, int part) : it(prm, prefix, seqlens, part), base(0) { valid = it.next(u); }
+  __device__ Cursor(const DecodeParams& prm, const int* prefix, const int* seqlens, int part) : it(prm, prefix, seqlens, part), base(0), ord(0) { valid = it.next(u); }
   __device__ bool locate(int k, int& local) {
-    while (valid && k >= base + (u.t1 - u.t0)) { base += u.t1 - u.t0; valid = it.next(u); }
+    while (valid && k >= base + (u.t1 - u.t0)) { base += u.t1 - u.t0; valid = it.next(u); ++ord; }
     local = k - base;
     return valid;
   }
@@ -188,24 +189,35 @@ __device__ __forceinline__ void prefetch_q_row(const DecodeParams& prm, const Un
   }
 }
 
-// One query row: four 64-column blocks [blk0, blk0 + 4) of its latent part, global memory -> tensor memory.
-__device__ __forceinline__ void load_q_latent(const uint4* qrow, bool valid, int blk0, uint32_t taddr) {
-#pragma unroll 1
-  for (int b = blk0; b < blk0 + 4; b += 2) {
-    uint32_t x0[32], x1[32];
-    if (valid) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        ldg_256(qrow + b * 8 + 2 * c, x0, 8 * c);
-        ldg_256(qrow + b * 8 + 8 + 2 * c, x1, 8 * c);
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) { x0[i] = 0; x1[i] = 0; }
-    }
-    tmem_st_32x32b_x32(taddr + b * 32, x0);
-    tmem_st_32x32b_x32(taddr + b * 32 + 32, x1);
+// Q comes on chip through the K ring.  At the start of a unit every ring slot of a score CTA takes a piece of the
+// CTA's 128 Q rows as TMA boxes of 64 rows x one 64-column block ([row][128 B], 128-byte swizzle): slot s holds block
+// s (two boxes); the eight blocks of the latent part are two more than there are slots, so the four half-blocks of
+// blocks 6 and 7 ride in the spare third of slots 0-3; the RoPE block goes straight to its operand tile, counted on
+// slot 0's barrier.  The eight softmax warps then move the latent blocks into tensor memory, thread = row.
+constexpr uint32_t kQHalfBytes = 64 * 128;              // one box
+__device__ __forceinline__ void issue_q_piece(const CUtensorMap* q_map, uint32_t smem_base, uint32_t bars, int s, int row0) {
+  const uint32_t full = bars + 8u * (A_QFULL + s), dst = smem_base + kOffK + s * kKSlotBytes;
+  mbar_arrive_expect_tx(full, (s == 0 ? 5 : s < 4 ? 3 : 2) * kQHalfBytes);
+  tma_load_3d(dst, q_map, 0, row0, s, full);
+  tma_load_3d(dst + kQHalfBytes, q_map, 0, row0 + 64, s, full);
+  if (s < 4) tma_load_3d(dst + 2 * kQHalfBytes, q_map, 0, row0 + 64 * (s & 1), 6 + (s >> 1), full);
+  if (s == 0) {
+    tma_load_3d(smem_base + kOffQRope, q_map, 0, row0, 8, full);
+    tma_load_3d(smem_base + kOffQRope + kQHalfBytes, q_map, 0, row0 + 64, 8, full);
   }
+}
+// 128 bytes of one row of a box (or of two stacked boxes) -> 32 tensor-memory columns (two bf16 per column)
+__device__ __forceinline__ void move_q_block(uint32_t box, int row, bool valid, uint32_t taddr) {
+  uint32_t x[32];
+#pragma unroll
+  for (int c = 0; c < 8; ++c)
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x[4 * c]), "=r"(x[4 * c + 1]), "=r"(x[4 * c + 2]), "=r"(x[4 * c + 3])
+                 : "r"(box + sw128_offset(row, c)));
+  if (!valid) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) x[i] = 0;
+  }
+  tmem_st_32x32b_x32(taddr, x);
 }
 
 struct RoleCtx {
@@ -413,7 +425,8 @@ __device__ __forceinline__ bool relay_phases(uint32_t bars, uint32_t lead_bars, 
 
 template <int kMode, bool kGuard>
 __global__ void __cluster_dims__(4, 1, 1) __launch_bounds__(kThreads, 1)
-decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const DecodeParams prm) {
+decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap q_map,
+                   const DecodeParams prm) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t smem_base = smem_u32(smem_raw);
   const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
@@ -454,6 +467,10 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       for (int i = 0; i < 4; ++i) mbar_init(bar(A_XCHG + i), 2);                        // the two warps that share 32 rows
       mbar_init(bar(A_QREADY), leader ? 9 : 8);                                         // 8 loading warps (+ relay)
       mbar_init(bar(A_QFREE), 1);
+      for (int i = 0; i < kNumKSlots; ++i) {
+        mbar_init(bar(A_QFULL + i), 1);
+        mbar_init(bar(A_QDONE + i), (i == 1 || i == 2) ? 6 : 4);     // the warps that read a piece of Q from slot i
+      }
     } else {
       for (int i = 0; i < kNumVSlots; ++i) { mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1); }
       for (int i = 0; i < kNumP; ++i) { mbar_init(bar(B_PFULL + i), 1); mbar_init(bar(B_OREADY + i), leader ? 9 : 8); }   // 8 correction warps (+ relay)
@@ -461,6 +478,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     fence_mbar_init();
     prefetch_tensormap(&k_map);
     prefetch_tensormap(&v_map);
+    prefetch_tensormap(&q_map);
   }
   if (wid == 5) { tmem_alloc_pair(tmem_slot, kTmemCols); tmem_relinquish_pair(); }
   tc_fence_before_sync();
@@ -508,10 +526,10 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
     __syncthreads();
     if (ps) { prefix = ps; seqlens = reinterpret_cast<const int*>(smem_raw + kOffSeqlens); }
   }
-  if (is_score && tid < kRowBlock) {   // the first unit's Q is on its way into L2 while the CTA sets itself up
+  if (is_score && tid < kNumKSlots) {   // the first unit's Q is requested before the roles start: one piece per lane
     UnitIter first(prm, prefix, seqlens, part);
     Unit fu;
-    if (first.next(fu)) prefetch_q_row(prm, fu, half * kRowBlock + tid);
+    if (first.next(fu)) issue_q_piece(&q_map, smem_base, bars, tid, fu.b * prm.R + fu.r0 + half * kRowBlock);
   }
 
   bool ok = true;
@@ -536,19 +554,31 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
         tc_fence_after_sync();
         if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 8 + 4 * un); };
         {
-          const int row = u.r0 + half * kRowBlock + qr;
-          const bool valid = row < prm.R;
-          const uint4* qrow = reinterpret_cast<const uint4*>(prm.q + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDqk);
-          load_q_latent(qrow, valid, grp_b ? 4 : 0, tbase + q_lane_base + kQCol);
-          if (grp_b) {
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-              const uint4 v = valid ? __ldg(qrow + 64 + cc) : make_uint4(0, 0, 0, 0);
-              st_shared_v4(smem_base + kOffQRope + sw128_offset(qr, cc), v.x, v.y, v.z, v.w);
-            }
+          // Group A moves blocks 0, 2, 4 (slots 0, 2, 4) and block 6, whose halves sit in slots 0 and 1; group B blocks
+          // 1, 3, 5 and block 7 (halves in slots 2 and 3).  A warp hands a slot back after its last read from it.
+          const bool valid = u.r0 + half * kRowBlock + qr < prm.R;
+          const int quarter = wid & 3;
+          const uint32_t kbase = smem_base + kOffK, trow = tbase + q_lane_base + kQCol, qpar = un & 1;
+          const uint32_t extra_col = 32 * (grp_b ? 7 : 6);
+#pragma unroll 1
+          for (int i = 0; i < 3 && ok; ++i) {
+            const int sl = 2 * i + (grp_b ? 1 : 0);
+            ok = warp_wait(bar(A_QFULL + sl), qpar);
+            if (!ok) break;
+            move_q_block(kbase + sl * kKSlotBytes, qr, valid, trow + 32 * sl);
+            if (grp_b ? (sl == 3 && quarter >= 2) : (sl == 0 && quarter < 2))
+              move_q_block(kbase + sl * kKSlotBytes + 2 * kQHalfBytes, qr & 63, valid, trow + extra_col);
+            warp_arrive(bar(A_QDONE + sl), lane);
+          }
+          if (!ok) break;
+          if (grp_b ? (quarter < 2) : (quarter >= 2)) {     // the half-block that rides in a slot of the other group
+            const int sl = grp_b ? 2 : 1;
+            ok = warp_wait(bar(A_QFULL + sl), qpar);
+            if (!ok) break;
+            move_q_block(kbase + sl * kKSlotBytes + 2 * kQHalfBytes, qr & 63, valid, trow + extra_col);
+            warp_arrive(bar(A_QDONE + sl), lane);
           }
           tmem_wait_st();
-          if (grp_b) fence_proxy_async_smem();
         }
         tc_fence_before_sync();
         warp_arrive(bar(A_QREADY), lane);
@@ -569,39 +599,68 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       // owns ring slot l and polls without blocking.  The bytes of both CTAs' halves are counted on the even CTA's
       // "full" barrier.  A sequence's last tile may have one page only: the odd CTA then loads the first page
       // again (finite values that the softmax masks as keys beyond the sequence).
+      // At the start of every unit the slot first carries the lane's piece of that unit's Q (see issue_q_piece; lane 0
+      // waits for the previous unit's MMAs to let go of the RoPE tile); the first unit's pieces were requested before
+      // the roles split.
       Cursor cur(prm, prefix, seqlens, part);
+      bool fin = lane >= kNumKSlots;
+      const bool first_out = !fin && cur.valid;
+      UnitIter qit = cur.it;                  // walks the units whose Q this lane has not requested (it stands behind the first)
+      Unit qu;
+      bool q_left = false, q_stale = first_out;
+      auto q_due = [&]() { if (q_stale) { q_left = qit.next(qu); q_stale = false; } return q_left; };
+      int q_ord = first_out ? 1 : 0;          // ordinal of the unit qu
+      int nq = first_out ? 1 : 0;             // pieces of Q requested for this slot
       int my_tile = lane / 3;                 // kNumKSlots = 6: lane l always loads column group l % 3, every second tile
       const int g = lane % 3;
       uint32_t par = 1;
-      bool fin = lane >= kNumKSlots, have = false;
+      int k_state = 0, k_ord = 0, pending = 0;   // K slot: 0 not looked up, 1 page number at hand, 2 none left; pending: 1 Q, 2 K
       int page_id = 0;
       int issued = 0;
-      const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane);
+      const uint32_t my_full = bar(A_KFULL + lane), my_empty = bar(A_KEMPTY + lane), my_qdone = bar(A_QDONE + lane);
       const uint32_t lead_full = lead_bars + 8u * (A_KFULL + lane);
       const uint32_t dst = smem_base + kOffK + lane * kKSlotBytes;
       uint64_t t_start = global_timer_ns();
       bool progress = false;
       for (uint32_t spin = 0;; ++spin) {
-        if (!fin && !have) {
-          int lt;
-          if (cur.locate(my_tile, lt)) {
-            const int t = cur.u.t0 + lt;
-            const int npg = (cur.u.n_b + kPage - 1) / kPage;
-            const int pg = (2 * t + half < npg) ? 2 * t + half : 2 * t;
-            page_id = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + pg);
-            have = true;
-          } else {
-            fin = true;
+        if (!fin && pending == 0) {
+          if (k_state == 0) {
+            int lt;
+            if (cur.locate(my_tile, lt)) {
+              const int t = cur.u.t0 + lt;
+              const int npg = (cur.u.n_b + kPage - 1) / kPage;
+              const int pg = (2 * t + half < npg) ? 2 * t + half : 2 * t;
+              page_id = __ldg(prm.block_table + static_cast<size_t>(cur.u.b) * prm.max_blocks_per_seq + pg);
+              k_ord = cur.ord;
+              k_state = 1;
+            } else {
+              k_state = 2;
+            }
           }
+          if ((k_state == 2 || q_ord <= k_ord) && q_due()) pending = 1;
+          else if (k_state == 1) pending = 2;
+          else fin = true;
         }
-        if (have && mbar_probe(my_empty, par)) {
-          if (leader) mbar_arrive_expect_tx(my_full, 2 * kKSlotBytes);
-          tma_load_4d_pair(dst, &k_map, 0, 0, 3 * g, page_id * 8, lead_full);
-          my_tile += 2;
-          par ^= 1;
-          ++issued;
-          have = false;
-          progress = true;
+        if (pending != 0) {
+          // the slot is free when its last K load has been used up by the MMAs and its last piece of Q has been moved
+          bool free_now = mbar_probe(my_empty, par) && (nq == 0 || mbar_probe(my_qdone, (nq - 1) & 1));
+          if (free_now && pending == 1 && lane == 0 && q_ord > 0) free_now = mbar_probe(bar(A_QFREE), (q_ord - 1) & 1);
+          if (free_now) {
+            if (pending == 1) {
+              issue_q_piece(&q_map, smem_base, bars, lane, qu.b * prm.R + qu.r0 + half * kRowBlock);
+              q_stale = true;
+              ++q_ord; ++nq;
+            } else {
+              if (leader) mbar_arrive_expect_tx(my_full, 2 * kKSlotBytes);
+              tma_load_4d_pair(dst, &k_map, 0, 0, 3 * g, page_id * 8, lead_full);
+              my_tile += 2;
+              par ^= 1;
+              ++issued;
+              k_state = 0;
+            }
+            pending = 0;
+            progress = true;
+          }
         }
         if (__all_sync(0xffffffffu, fin)) break;
         const bool any_progress = __any_sync(0xffffffffu, progress);
@@ -612,6 +671,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
       if (!ok) {
         if (lane == 0) report_timeout(prm.status);
         if (leader && issued > 0 && lane < kNumKSlots) mbar_wait(my_full, (issued - 1) & 1);   // let copies in flight land
+        if (nq > 0 && lane < kNumKSlots) mbar_wait(bar(A_QFULL + lane), (nq - 1) & 1);
       }
     } else if (wid == 5) {
       // ---- MMA issuer (even CTA only): S[sb] = Q K^T for both CTAs' rows, 36 steps of K = 16 over three slots
@@ -994,7 +1054,7 @@ cudaError_t prepare_variant(int device) {
 }
 
 template <int kMode, bool kGuard>
-cudaError_t launch_variant(const CUtensorMap& kmap, const CUtensorMap& vmap, const DecodeParams& prm, cudaStream_t stream) {
+cudaError_t launch_variant(const CUtensorMap& kmap, const CUtensorMap& vmap, const CUtensorMap& qmap, const DecodeParams& prm, cudaStream_t stream) {
   int device = 0;
   cudaError_t err = cudaGetDevice(&device);
   if (err != cudaSuccess) return err;
@@ -1003,7 +1063,7 @@ cudaError_t launch_variant(const CUtensorMap& kmap, const CUtensorMap& vmap, con
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
   fill_config(cfg, attr, prm.P, stream);
-  return cudaLaunchKernelEx(&cfg, decode_quad_kernel<kMode, kGuard>, kmap, vmap, prm);
+  return cudaLaunchKernelEx(&cfg, decode_quad_kernel<kMode, kGuard>, kmap, vmap, qmap, prm);
 }
 
 }  // namespace
@@ -1058,11 +1118,25 @@ cudaError_t launch_decode_quad(const DecodeParams& prm, cudaStream_t stream, int
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (vr != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
+  // Q: (64 columns, rows of all sequences, 9 column blocks); one box = 64 rows x one column block, laid out
+  // [row][64 columns] like an operand tile.  Rows past the end of the array read as zero; rows of a following
+  // sequence that a short block's boxes cover are dropped by the kernel.
+  CUtensorMap qmap;
+  {
+    const cuuint64_t qdims[3] = {64, static_cast<cuuint64_t>(prm.B) * prm.R, static_cast<cuuint64_t>(kDqk / 64)};
+    const cuuint64_t qstrides[2] = {static_cast<cuuint64_t>(kDqk) * 2, 128};
+    const cuuint32_t qbox[3] = {64, 64, 1};
+    const cuuint32_t qestr[3] = {1, 1, 1};
+    const CUresult qr = encode(&qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(prm.q), qdims, qstrides,
+                               qbox, qestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (qr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
   const int mode = prm.flags & 3;
   const bool guard = !(prm.flags & 4);
-  if (mode == 0) return guard ? launch_variant<0, true>(kmap, vmap, prm, stream) : launch_variant<0, false>(kmap, vmap, prm, stream);
-  if (mode == 1) return guard ? launch_variant<1, true>(kmap, vmap, prm, stream) : launch_variant<1, false>(kmap, vmap, prm, stream);
-  return launch_variant<2, true>(kmap, vmap, prm, stream);
+  if (mode == 0) return guard ? launch_variant<0, true>(kmap, vmap, qmap, prm, stream) : launch_variant<0, false>(kmap, vmap, qmap, prm, stream);
+  if (mode == 1) return guard ? launch_variant<1, true>(kmap, vmap, qmap, prm, stream) : launch_variant<1, false>(kmap, vmap, qmap, prm, stream);
+  return launch_variant<2, true>(kmap, vmap, qmap, prm, stream);
 }
 
 }  // namespace amla
