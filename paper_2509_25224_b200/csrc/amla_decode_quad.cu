@@ -24,6 +24,7 @@
 
 #include "amla_common.cuh"
 #include "amla_sm100.cuh"
+#include "amla_epilogue.cuh"
 
 namespace amla {
 
@@ -72,7 +73,7 @@ constexpr uint32_t kOffSeqlens = kOffPlan + ((kSmemPlanItems + 1) * 4 + 15) / 16
 #ifdef AMLA_TRACE
 // trace builds: every CTA keeps its stamps (low 32 bits of its SM's cycle counter) in shared memory, so that taking
 // one does not put a global store in front of the role's next release, and dumps them when it is done
-constexpr int kQTraceEvents = 16, kQTraceIdx = 11;
+constexpr int kQTraceEvents = 16, kQTraceIdx = 10;
 constexpr uint32_t kOffTrace = kOffSeqlens + kSmemPlanItems * 4;
 constexpr uint32_t kSmemBytes = kOffTrace + kQTraceEvents * kQTraceIdx * 4;
 #define QSTAMP(smem_base_, ev, idx)                                                                          \
@@ -826,10 +827,11 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
         // chunks each, scale them and store them from registers with 256-bit stores (a full 32-byte sector per lane).
         {
           const uint32_t gl = gt - 1;
+          if (tid == 0) QSTAMP(smem_base, 14, un);
           ok = warp_wait(bar(X_PV + gl % kNumP), (gl / kNumP) & 1);
           if (!ok) break;
           tc_fence_after_sync();
-          if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 10 + 4 * un); };
+          if (tid == 0) { QSTAMP(smem_base, 12, un); if (un < 1) QSTAMP_NS(smem_base, 3); };
           const int row = u.r0 + half * kRowBlock + r;               // this thread's row within the sequence
           const bool valid = row < prm.R;
           __nv_bfloat16* orow = prm.out + (static_cast<size_t>(u.b) * prm.R + (valid ? row : 0)) * kDv;
@@ -845,30 +847,19 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
               tmem_wait_ld();
               if (cq + e + 1 < 8) tmem_ld_32x32b_x32(tbase + lane_base + 32 * (c_first + cq + e + 1), o[e ^ 1]);
               const int cc = c_first + cq + e;
+              uint32_t w[16];
+              uint16_t* dst;
               if (slot < 0) {
-                uint32_t w[16];
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj)
-                  w[jj] = pack_bf16x2(__uint_as_float(o[e][2 * jj]) * inv, __uint_as_float(o[e][2 * jj + 1]) * inv);
-                if (valid) {
-                  stg_256(orow + 32 * cc, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
-                  stg_256(orow + 32 * cc + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
-                }
+                epilogue_chunk_bf16(o[e], inv, w);
+                dst = reinterpret_cast<uint16_t*>(orow) + 32 * cc;
               } else {
-                // split unit: half precision with the chunk's power-of-two scale (see "Split partials")
-                float x[32], mx = 0.f;
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) { x[jj] = __uint_as_float(o[e][jj]) * inv; mx = fmaxf(mx, fabsf(x[jj])); }
-                float f;
-                const uint32_t sb = partial_scale_byte(mx, &f);
+                const uint32_t sb = epilogue_chunk_partial(o[e], inv, w);
                 if (cq + e < 4) sc_lo |= sb << (8 * (cq + e)); else sc_hi |= sb << (8 * (cq + e - 4));
-                uint32_t w[16];
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) w[jj] = pack_f16x2(x[2 * jj] * f, x[2 * jj + 1] * f);
-                if (valid) {
-                  stg_256(hrow + 32 * cc, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
-                  stg_256(hrow + 32 * cc + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
-                }
+                dst = hrow + 32 * cc;
+              }
+              if (valid) {
+                stg_256(dst, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                stg_256(dst + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
               }
             }
           }
@@ -879,7 +870,7 @@ decode_quad_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_const
             else prm.part_lse[prow] = lse;
           }
           tc_fence_before_sync();
-          if (tid == 0) { if (un < 1) QSTAMP_NS(smem_base, 11 + 4 * un); };
+          if (tid == 0) QSTAMP(smem_base, 13, un);
         }
         ++un;
       }
