@@ -171,12 +171,6 @@ __device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint3
       ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(cluster_bar)
       : "memory");
 }
-// 256-bit read-only global load (32-byte aligned address).
-__device__ __forceinline__ void ldg_256(const void* p, uint32_t (&r)[32], int at) {
-  asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[at]), "=r"(r[at + 1]), "=r"(r[at + 2]), "=r"(r[at + 3]), "=r"(r[at + 4]), "=r"(r[at + 5]), "=r"(r[at + 6]), "=r"(r[at + 7])
-               : "l"(p));
-}
 // 256-bit global store (32-byte aligned address).
 __device__ __forceinline__ void stg_256(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e, uint32_t f, uint32_t g, uint32_t h) {
   asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
