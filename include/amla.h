@@ -87,6 +87,9 @@ int amla_mla_decode_workspace_size(int B, int Sq, int H, int max_blocks_per_seq,
  *                beyond the sequence length must hold finite values (they are multiplied by zero).
  *   block_table  device, int32 [B, max_blocks_per_seq]; entries beyond ceil(seqlens[b]/64) are ignored
  *   seqlens      device, int32 [B], 0 <= seqlens[b] <= 64 * max_blocks_per_seq
+ *                (read while the kernel in front on the stream may still be draining if that kernel is one of
+ *                this library's own, which never write it; a caller's kernel that produces seqlens must not itself
+ *                release its dependents early by programmatic dependent launch)
  *   out          device, bf16 [B, Sq, H, 512], 16-byte aligned
  *   lse          device, fp32 [B, Sq, H], natural logarithm
  *   workspace    device, 256-byte aligned, at least amla_mla_decode_workspace_size() bytes; contents
